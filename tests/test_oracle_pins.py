@@ -1,0 +1,442 @@
+"""Pins of the CPU oracle against things other than itself: library routines, closed forms,
+brute force, invariants, hand-worked vectors and the numbers the paper prints."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+from oracle import feplb_oracle as O
+from paper_2604_19654_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _kv(path):
+    out = {}
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if "=" in line:
+            k, v = line.split("=", 1)
+            out[k.strip()] = v.strip()
+    return out
+
+
+# ----------------------------------------------------------------------------- paper numbers
+
+def test_paper_expert_size_and_buffer():
+    g = _kv(os.path.join(GOLDEN, "paper_numbers.txt"))
+    w = W.get_workload("cfg3")
+    expert_bytes = 3 * w.d * w.f * 2                       # W1, W3, W2 in bf16
+    assert expert_bytes == int(g["expert_mib"]) * 2 ** 20   # Section 2.3: 72 MiB per expert
+    assert int(g["max_num_dyn"]) * int(g["expert_mib"]) == int(g["buffer_mib"])
+    assert int(g["buffer_mib"]) * 2 ** 20 / (int(g["hbm_gb"]) * 2 ** 30) < float(g["buffer_frac_below"]) + 1e-4
+    assert w.E == int(g["experts"]) and w.E // 8 == int(g["experts_per_device_ep8"])
+    assert w.L - w.dyn == int(g["static_per_device_dyn4"])
+
+
+def test_paper_straggler_tables_arithmetic():
+    """token_straggler is max - mean; the reductions printed in Tables 3 and 4 follow from the
+    printed before/after values."""
+    g = _kv(os.path.join(GOLDEN, "paper_numbers.txt"))
+    for key in ("table3", "table4"):
+        for row in g[key].split(";"):
+            _, before, after, pct = row.split()
+            assert round(100 * (1 - float(after) / float(before))) == int(pct)
+    # a load vector whose max - mean is the Table 3 value: mean 10000, max 10000 + 6666
+    load = [10000 + 6666, 10000 - 6666 / 7.0] + [10000 - 6666 / 7.0] * 6
+    assert O.token_straggler(load) == pytest.approx(6666)
+    assert O.straggler_ratio(load) == pytest.approx(1.6666)
+
+
+# ----------------------------------------------------------------------------- histogram
+
+@settings(max_examples=50, deadline=None)
+@given(st.integers(1, 6), st.integers(1, 64), st.integers(1, 4), st.integers(0, 2 ** 31))
+def test_hist_matches_bincount(r, t, k, seed):
+    E = r * 3
+    rng = np.random.default_rng(seed)
+    ids = rng.integers(0, E, size=(t, k)).astype(np.int32)
+    counts, load = O.route_hist(ids, E, r)
+    assert np.array_equal(counts, np.bincount(ids.ravel(), minlength=E))
+    assert counts.sum() == t * k == load.sum()               # token conservation
+    assert np.array_equal(load, counts.reshape(r, 3).sum(1))
+
+
+def test_hist_rejects_out_of_range():
+    with pytest.raises(ValueError):
+        O.route_hist(np.array([[0, 8]]), 8, 2)
+    with pytest.raises(ValueError):
+        O.route_hist(np.array([[-1, 0]]), 8, 2)
+
+
+# ----------------------------------------------------------------------------- permutation
+
+@settings(max_examples=50, deadline=None)
+@given(st.integers(1, 12), st.integers(0, 80), st.integers(1, 4), st.sampled_from([1, 8, 128]),
+       st.integers(0, 2 ** 31))
+def test_permute_invariants_and_argsort(E, t, k, A, seed):
+    rng = np.random.default_rng(seed)
+    ids = rng.integers(0, E, size=(t, k)).astype(np.int32)
+    s2r, r2t, pad_off, S_pad = O.permute(ids, E, A)
+    counts = np.bincount(ids.ravel(), minlength=E)
+    # every (token, k) slot placed exactly once
+    flat = s2r.ravel()
+    assert len(set(flat.tolist())) == t * k
+    assert np.array_equal(np.sort(flat), np.flatnonzero(r2t >= 0))
+    assert S_pad == sum(O.round_up(int(c), A) for c in counts)
+    for s, row in enumerate(flat.tolist()):
+        e = ids.ravel()[s]
+        assert pad_off[e] <= row < pad_off[e] + counts[e]   # lands in its expert's segment
+        assert r2t[row] == s // k
+    # stability: rows of one expert appear in increasing slot order
+    for e in range(E):
+        rows = flat[ids.ravel() == e]
+        assert np.all(np.diff(rows) == 1) if rows.size > 1 else True
+    if A == 1 and t * k:
+        order = np.argsort(ids.ravel(), kind="stable")       # library stable sort
+        inv = np.empty_like(order)
+        inv[order] = np.arange(order.size)
+        assert np.array_equal(flat, inv)
+
+
+def test_permute_bruteforce_tiny():
+    ids = np.array([[2, 0], [0, 2], [1, 0]], np.int32)       # slots: 2 0 0 2 1 0
+    s2r, r2t, pad_off, S_pad = O.permute(ids, 3, 1)
+    assert s2r.ravel().tolist() == [4, 0, 1, 5, 3, 2]
+    assert r2t.tolist() == [0, 1, 2, 2, 0, 1]
+    assert pad_off.tolist() == [0, 3, 4] and S_pad == 6
+    s2r, r2t, pad_off, S_pad = O.permute(ids, 3, 4)
+    assert pad_off.tolist() == [0, 4, 8] and S_pad == 12
+    assert s2r.ravel().tolist() == [8, 0, 1, 9, 4, 2]
+    assert r2t.tolist() == [0, 1, 2, -1, 2, -1, -1, -1, 0, 1, -1, -1]
+
+
+def test_gather_rows_roundtrip():
+    rng = np.random.default_rng(0)
+    x = rng.integers(0, 2 ** 16, size=(5, 7)).astype(np.uint16)
+    ids = rng.integers(0, 4, size=(5, 3)).astype(np.int32)
+    s2r, r2t, _, S_pad = O.permute(ids, 4, 8)
+    xp = O.gather_rows(x, r2t)
+    assert xp.shape == (S_pad, 7)
+    for t in range(5):
+        for k in range(3):
+            assert np.array_equal(xp[s2r[t, k]], x[t])
+    assert not xp[r2t < 0].any()
+
+
+# ----------------------------------------------------------------------------- plan
+
+def _load_cases():
+    cases, cur = [], None
+    for line in open(os.path.join(GOLDEN, "plan_handworked.txt")):
+        line = line.split("#")[0].rstrip("\n")
+        if "=" not in line:
+            continue
+        k, v = [s.strip() for s in line.split("=", 1)]
+        if k == "case":
+            cur = {"case": v}
+            cases.append(cur)
+        else:
+            cur[k] = v
+    return cases
+
+
+@pytest.mark.parametrize("c", _load_cases(), ids=lambda c: c["case"])
+def test_plan_handworked(c):
+    R, L = int(c["R"]), int(c["L"])
+    counts = [int(v) for v in c["counts"].split()]
+    mask = [int(v) for v in c["mask"].split()]
+    p = O.plan(counts, mask, R, tau=int(c["tau"]), max_num_dyn=int(c["max_num_dyn"]),
+               ranks_per_domain=int(c["domain"]),
+               policy=O.POLICY_LITERAL if c["policy"] == "literal" else O.POLICY_FIRST_FIT,
+               split=int(c["split"]), split_granule=int(c["g"]))
+    exp_moves = []
+    for m in c["moves"].split():
+        e, sd, rows = m.split(":")
+        s, dd = sd.split(">")
+        exp_moves.append((int(e), int(s), int(dd), int(rows)))
+    assert p["moves"] == exp_moves
+    assert p["load_before"].tolist() == [int(v) for v in c["load_before"].split()]
+    assert p["load_after"].tolist() == [int(v) for v in c["load_after"].split()]
+    assert len(counts) == R * L
+
+
+def _check_plan_invariants(counts, mask, R, p, tau, max_num_dyn, D, split, g, A=1):
+    E = len(counts)
+    L = E // R
+    D = D or R
+    counts = np.asarray(counts)
+    before = counts.reshape(R, L).sum(1)
+    assert np.array_equal(p["load_before"], before)
+    assert p["load_after"].sum() == before.sum() == counts.sum()      # conservation
+    for dom in range(R // D):
+        sl = slice(dom * D, (dom + 1) * D)
+        assert p["load_after"][sl].sum() == before[sl].sum()           # nothing crosses a domain
+        assert p["load_after"][sl].max() <= before[sl].max()           # max load never rises
+    recv = np.zeros(R, int)
+    seen_pairs = set()
+    moved_rows = np.zeros(E, int)
+    for (e, src, dst, rows) in p["moves"]:
+        assert mask[e] and src == e // L and dst != src
+        assert src // D == dst // D
+        assert rows >= max(tau, 1)
+        recv[dst] += 1
+        assert (e, dst) not in seen_pairs
+        seen_pairs.add((e, dst))
+        moved_rows[e] += rows
+        if not split:
+            assert rows == counts[e]
+        elif moved_rows[e] < counts[e]:
+            assert rows % g == 0
+    assert np.all(moved_rows <= counts)
+    assert np.all(recv <= max_num_dyn)
+    if not split:
+        assert len({m[0] for m in p["moves"]}) == len(p["moves"])     # an expert moves at most once
+    # groups tile each expert's segment exactly once, in expert order
+    pad_off, _ = O.segment_offsets(counts, A)
+    per_e = np.zeros(E, int)
+    last_e = -1
+    nxt = {}
+    for (e, row_start, rows, exec_rank, is_dyn) in p["groups"]:
+        assert e >= last_e and rows > 0 and is_dyn == int(bool(mask[e]))
+        last_e = e
+        assert row_start == nxt.get(e, int(pad_off[e]))
+        nxt[e] = row_start + rows
+        per_e[e] += rows
+        if not mask[e]:
+            assert exec_rank == e // L
+    assert np.array_equal(per_e, counts)
+    assert np.array_equal(p["exec_rows"].sum(0), counts)
+    assert np.array_equal(p["exec_rows"].sum(1), p["load_after"])
+    # replaying the moves reproduces load_after, and in whole mode every accepted move had rows < gap
+    load = before.astype(np.int64).copy()
+    for (e, src, dst, rows) in p["moves"]:
+        if not split:
+            assert rows < load[src] - load[dst]
+        load[src] -= rows
+        load[dst] += rows
+    assert np.array_equal(load, p["load_after"])
+
+
+plan_inputs = st.tuples(
+    st.sampled_from([1, 2, 3, 4, 8]), st.integers(1, 6), st.integers(0, 2 ** 31),
+    st.sampled_from([0, 1, 5, 40]), st.integers(0, 4), st.sampled_from([0, 1]),
+    st.sampled_from([0, 1]), st.sampled_from([1, 16, 128]), st.booleans())
+
+
+@settings(max_examples=300, deadline=None)
+@given(plan_inputs)
+def test_plan_invariants(args):
+    R, L, seed, tau, mnd, policy, split, g, use_dom = args
+    rng = np.random.default_rng(seed)
+    E = R * L
+    scale = rng.choice([4, 60, 2000])
+    counts = (rng.dirichlet(np.full(E, 0.3)) * scale * E).astype(np.int64)
+    mask = (rng.random(E) < 0.6).astype(np.uint8)
+    D = 0
+    if use_dom and R % 2 == 0:
+        D = 2
+    kw = dict(tau=tau, max_num_dyn=mnd, ranks_per_domain=D, policy=policy, split=split, split_granule=g)
+    p = O.plan(counts, mask, R, **kw)
+    _check_plan_invariants(counts, mask, R, p, tau, mnd, D, split, g)
+    q = O.plan(counts.copy(), mask.copy(), R, **kw)                  # pure function
+    assert p["moves"] == q["moves"] and p["groups"] == q["groups"]
+    if split:
+        M = -(-int(counts.sum()) // R) if not D else None
+        if M is not None:
+            for r in range(R):      # no rank is pushed across the mean: receivers stay <= M, donors >= M
+                if p["load_after"][r] > p["load_before"][r]:
+                    assert p["load_after"][r] <= M
+                if p["load_after"][r] < p["load_before"][r]:
+                    assert p["load_after"][r] >= M
+
+
+def test_plan_closed_form_special_cases():
+    counts = np.array([50, 10, 3, 7, 100, 20, 1, 9])
+    full = np.ones(8, np.uint8)
+    # R = 1, empty mask, tau above every count, no receive slots: nothing can move
+    for kw, R, mask in [({}, 1, full), ({}, 2, np.zeros(8, np.uint8)), ({"tau": 101}, 2, full),
+                        ({"max_num_dyn": 0}, 2, full)]:
+        p = O.plan(counts, mask, R, **kw)
+        assert p["moves"] == [] and np.array_equal(p["load_after"], p["load_before"])
+        assert [g_[0] for g_ in p["groups"]] == list(range(8))
+    # all counts equal: loads equal, gap 0
+    p = O.plan(np.full(8, 5), full, 4)
+    assert p["moves"] == []
+
+
+def test_plan_one_hot_expert_exact():
+    # loads [100, 10, 10]; hot expert 0 has 60 rows < gap 90 -> one move to rank 1 (lowest id of the two minima)
+    counts = np.array([60, 40, 10, 0, 10, 0])
+    mask = np.array([1, 0, 0, 0, 0, 0], np.uint8)
+    p = O.plan(counts, mask, 3, tau=1)
+    assert p["moves"] == [(0, 0, 1, 60)]
+    assert p["load_after"].tolist() == [40, 70, 10]
+    # a hot expert at least as large as the gap stays (moving it cannot lower the maximum)
+    counts = np.array([95, 5, 10, 0, 10, 0])
+    p = O.plan(counts, mask, 3, tau=1)
+    assert p["moves"] == []
+
+
+def _brute_force_best_max(counts, mask, R, max_num_dyn):
+    """Smallest achievable max load over all placements of whole dynamic experts."""
+    E = len(counts)
+    L = E // R
+    dyn = [e for e in range(E) if mask[e]]
+    base = [0] * R
+    for e in range(E):
+        if not mask[e]:
+            base[e // L] += counts[e]
+    best = None
+    for assign in itertools.product(range(R), repeat=len(dyn)):
+        recv = [0] * R
+        load = list(base)
+        for e, r in zip(dyn, assign):
+            load[r] += counts[e]
+            if r != e // L:
+                recv[r] += 1
+        if max(recv) > max_num_dyn:
+            continue
+        m = max(load)
+        best = m if best is None else min(best, m)
+    return best
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.sampled_from([(2, 2), (2, 3), (3, 2), (2, 4)]), st.integers(0, 2 ** 31), st.sampled_from([0, 1]))
+def test_plan_bruteforce_bound(shape, seed, policy):
+    R, L = shape
+    rng = np.random.default_rng(seed)
+    E = R * L
+    counts = rng.integers(0, 50, size=E)
+    mask = (rng.random(E) < 0.7).astype(np.uint8)
+    p = O.plan(counts, mask, R, tau=1, max_num_dyn=3, policy=policy)
+    best = _brute_force_best_max(counts.tolist(), mask.tolist(), R, 3)
+    assert best <= p["load_after"].max() <= p["load_before"].max()
+
+
+def test_select_dynamic():
+    score = [5, 9, 9, 1, 0, 0, 3, 2]
+    m = O.select_dynamic(score, 8, 2, 2)
+    assert m.tolist() == [0, 1, 1, 0, 0, 0, 1, 1]          # rank 0: e1, e2; rank 1: e6 (3), e7 (2)
+    assert O.select_dynamic([1, 1, 1, 1], 4, 1, 2).tolist() == [1, 1, 0, 0]   # ties -> lower id
+    assert O.select_dynamic(score, 8, 2, 0).sum() == 0
+    assert O.select_dynamic(score, 8, 2, 9).sum() == 8
+
+
+def test_plan_improves_every_workload():
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+        w = W.get_workload(name)
+        ids, _ = W.gen_routing(w, 0)
+        counts, load = O.route_hist(ids, w.E, w.R)
+        mask = O.select_dynamic(counts, w.E, w.R, w.dyn)
+        for split in (0, 1):
+            g = 16 if name == "cfg1" else 128
+            p = O.plan(counts, mask, w.R, w.tau, w.max_num_dyn, split=split, split_granule=g)
+            assert O.straggler_ratio(p["load_after"]) < O.straggler_ratio(load)
+            _check_plan_invariants(counts, mask, w.R, p, w.tau, w.max_num_dyn, 0, split, g)
+
+
+# ----------------------------------------------------------------------------- expert FFN
+
+def _bits(a):
+    return W.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def test_silu_closed_forms():
+    z = np.array([-3.0, -1.0, 0.0, 0.5, 2.0, 30.0])
+    s = O.silu(z)
+    assert s[2] == 0.0
+    assert np.allclose(s - O.silu(-z), z)                    # silu(z) - silu(-z) = z
+    assert s[1] == pytest.approx(-1.0 / (1.0 + math.e))
+    assert s[5] == pytest.approx(30.0, rel=1e-12)
+    assert np.allclose(s, z * 0.5 * (1.0 + np.tanh(z / 2.0)))   # sigmoid written via tanh
+
+
+def test_ffn_against_scalar_loops():
+    rng = np.random.default_rng(3)
+    E, d, f, n = 3, 5, 4, 7                                   # non-square on purpose
+    x = _bits(rng.standard_normal((n, d)))
+    w1 = _bits(rng.standard_normal((E, f, d)))
+    w3 = _bits(rng.standard_normal((E, f, d)))
+    w2 = _bits(rng.standard_normal((E, d, f)))
+    re = np.array([2, 0, 1, 1, -1, 0, 2])
+    y = O.expert_ffn(x, re, w1, w3, w2)
+    X, W1, W3, W2 = (W.bf16_bits_to_f64(a) for a in (x, w1, w3, w2))
+    for i in range(n):
+        e = re[i]
+        if e < 0:
+            assert not y[i].any()
+            continue
+        h = []
+        for c in range(f):
+            a = sum(X[i, j] * W1[e, c, j] for j in range(d))
+            b = sum(X[i, j] * W3[e, c, j] for j in range(d))
+            h.append(a / (1.0 + math.exp(-a)) * b)
+        for o in range(d):
+            ref = sum(h[c] * W2[e, o, c] for c in range(f))
+            assert y[i, o] == pytest.approx(ref, rel=1e-12, abs=1e-15)
+
+
+def test_ffn_one_hot_rows_and_linearity():
+    rng = np.random.default_rng(4)
+    E, d, f = 2, 6, 3
+    w1 = _bits(rng.standard_normal((E, f, d)))
+    w3 = _bits(rng.standard_normal((E, f, d)))
+    w2 = _bits(rng.standard_normal((E, d, f)))
+    W1, W3, W2 = (W.bf16_bits_to_f64(a) for a in (w1, w3, w2))
+    x = _bits(np.eye(d))                                       # row i = unit vector i
+    for e in range(E):
+        y = O.expert_ffn(x, np.full(d, e), w1, w3, w2)
+        for i in range(d):
+            h = O.silu(W1[e, :, i]) * W3[e, :, i]              # x W1 picks column i of the d x f matrix
+            assert np.allclose(y[i], W2[e] @ h, rtol=1e-12)
+    # doubling W2 doubles y; W3 = 0 gives 0
+    xr = _bits(rng.standard_normal((4, d)))
+    y1 = O.expert_ffn(xr, np.zeros(4, int), w1, w3, w2)
+    y2 = O.expert_ffn(xr, np.zeros(4, int), w1, w3, _bits(2 * W.bf16_bits_to_f32(w2)))
+    assert np.allclose(y2, 2 * y1, rtol=1e-12)
+    assert not O.expert_ffn(xr, np.zeros(4, int), w1, np.zeros_like(w3), w2).any()
+
+
+# ----------------------------------------------------------------------------- combine, whole layer
+
+def test_combine_scalar_loops_and_identity_roundtrip():
+    rng = np.random.default_rng(5)
+    T, K, d, E = 6, 3, 4, 5
+    ids = rng.integers(0, E, size=(T, K)).astype(np.int32)
+    s2r, r2t, _, S_pad = O.permute(ids, E, 8)
+    y = rng.standard_normal((S_pad, d))
+    g = rng.random((T, K)).astype(np.float32)
+    out = O.combine(y, s2r, g)
+    for t in range(T):
+        for j in range(d):
+            assert out[t, j] == pytest.approx(sum(float(g[t, k]) * y[s2r[t, k], j] for k in range(K)), rel=1e-13)
+    # K = 1, gate = 1, identity "FFN": dispatch then combine returns x exactly
+    ids1 = rng.integers(0, E, size=(T, 1)).astype(np.int32)
+    x = _bits(rng.standard_normal((T, d)))
+    s2r1, r2t1, _, _ = O.permute(ids1, E, 1)
+    xp = O.gather_rows(x, r2t1)
+    out1 = O.combine(W.bf16_bits_to_f64(xp), s2r1, np.ones((T, 1), np.float32))
+    assert np.array_equal(out1, W.bf16_bits_to_f64(x))
+
+
+def test_staged_pipeline_equals_layer_definition():
+    """permute -> gather -> FFN on permuted rows -> combine equals sum_k g * FFN_e(x_t), with or
+    without padding, and whatever the plan says (the plan only relabels ranks)."""
+    w = W.get_workload("cfg1")
+    x, ids, gates = W.gen_microbatch(w, 0)
+    w1, w3, w2 = W.gen_weights(w)
+    ref = O.moe_layer(x, ids, gates, w1, w3, w2, w.E)
+    for A in (1, 128):
+        s2r, r2t, _, S_pad = O.permute(ids, w.E, A)
+        xp = O.gather_rows(x, r2t)
+        re = O.row_experts(ids, s2r, S_pad)
+        y = O.expert_ffn(xp, re, w1, w3, w2)
+        out = O.combine(y, s2r, gates)
+        assert np.allclose(out, ref, rtol=1e-12, atol=1e-18)
+    sub = np.array([0, 17, 255])
+    assert np.allclose(O.moe_layer(x, ids, gates, w1, w3, w2, w.E, tokens=sub), ref[sub], rtol=1e-12, atol=1e-18)
