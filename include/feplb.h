@@ -1,0 +1,240 @@
+/*
+ * feplb.h -- C ABI of libfeplb: the per-micro-batch MoE-layer hot path of FEPLB on one
+ * NVIDIA B200 (sm_100a), with the expert-parallel layout modelled as R virtual ranks.
+ *
+ * Path (paper Section 2.3, per-micro-batch timeline):
+ *   router output (given)  ->  feplb_route_hist   per-expert token counts        (Section 2.2)
+ *                          ->  feplb_plan         greedy rebalancing plan (host) (Section 2.3)
+ *                          ->  feplb_dispatch     permutation into expert-contiguous rows (2.2)
+ *                          ->  feplb_expert_ffn   static, then dynamic grouped SwiGLU GEMMs (2.3)
+ *                          ->  feplb_combine      gate-weighted return of the results    (2.3)
+ *   feplb_moe_forward runs the whole path and overlaps the host planner with the static-expert
+ *   GEMM, as the paper's timeline does.
+ *
+ * Notation: T tokens, K experts per token, E experts, R ranks, L = E/R experts per rank in
+ * contiguous blocks (home(e) = e / L), S = T*K slots with slot s = t*K + k, d hidden size,
+ * f expert width, A = row_align, S_cap = feplb_s_pad(cfg) rows of the permuted buffers.
+ *
+ * Conventions
+ *   - Every function returns 0 (FEPLB_OK) or a negative feplb_status; nothing throws.
+ *   - "dev" pointers are device global memory on the context's device, 16-byte aligned, owned
+ *     by the caller; "host" pointers are ordinary host memory.  The library keeps no pointer
+ *     after a call returns, except where stated (feplb_plan_async).
+ *   - Device work is enqueued on the cudaStream_t passed as `stream` (as void*) and is
+ *     asynchronous unless stated.  Calls on one context must not overlap on the GPU: they share
+ *     the context's scratch.
+ *   - bf16 tensors are row-major.  Expert weights are stored output-major:
+ *     w1, w3 [E, f, d] and w2 [E, d, f] (row n of w1[e] = the d coefficients of hidden unit n).
+ *   - Out-of-range expert ids and device-side waits that gave up are reported through the
+ *     context's status word: see feplb_check_status.  Kernels never trap.
+ *   - There is no CPU fallback: device entry points need a CUDA device of compute capability
+ *     10.0 and fail with FEPLB_E_CUDA otherwise.
+ */
+#ifndef FEPLB_H_
+#define FEPLB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FEPLB_OK = 0,
+  FEPLB_E_INVALID = -1, /* bad argument or unsupported shape */
+  FEPLB_E_RANGE = -2,   /* an expert id outside [0, E) was seen on the device */
+  FEPLB_E_CUDA = -3,    /* a CUDA runtime/driver call failed; text in feplb_last_error */
+  FEPLB_E_NOMEM = -4,   /* an allocation failed, or a caller-sized array is too small */
+  FEPLB_E_TIMEOUT = -5, /* a bounded host wait expired */
+  FEPLB_E_STATE = -6,   /* call order violated (e.g. plan_wait without plan_async) */
+  FEPLB_E_DEVICE = -7   /* a bounded device-side wait gave up, or counts disagree with ids */
+} feplb_status;
+
+enum { FEPLB_POLICY_LITERAL = 0, FEPLB_POLICY_FIRST_FIT = 1 };
+enum { FEPLB_MASK_GIVEN = 0, FEPLB_MASK_REACTIVE = 1 };
+enum { FEPLB_FFN_ALL = 0, FEPLB_FFN_STATIC = 1, FEPLB_FFN_DYNAMIC = 2 };
+
+/* Layer geometry and balancer parameters.
+ * Requirements: E % R == 0; d % 128 == 0; f % 64 == 0; 1 <= K <= 32; E <= 1024;
+ * row_align in {1, 128}; split_granule >= 1. */
+typedef struct {
+  int32_t T, K, E, R, d, f;
+  int32_t dyn;              /* dynamic experts per rank (Section 2.3), used by FEPLB_MASK_REACTIVE */
+  int32_t max_num_dyn;      /* received experts (pieces) per rank: the receive buffer holds
+                               max_num_dyn expert weights (Section 2.3, memory paragraph) */
+  int32_t tau;              /* minimum rows for a migration (Section 2.3, threshold tau) */
+  int32_t ranks_per_domain; /* ranks per NVLink domain, 0 = R (Section 2.2: rebalance only inside) */
+  int32_t policy;           /* FEPLB_POLICY_*: stop at, or skip, a busiest expert that does not fit */
+  int32_t split;            /* 0 = whole experts (the paper); 1 = cut hot experts (extension) */
+  int32_t split_granule;    /* rows; pieces of a cut expert are multiples of it */
+  int32_t row_align;        /* A: expert segments of the permuted buffers start at multiples of A */
+  int32_t mask_policy;      /* FEPLB_MASK_*: who chooses the dynamic experts in feplb_moe_forward */
+} feplb_config;
+
+/* One copy of the plan: `rows` rows of `expert` leave home rank `src` for rank `dst`. */
+typedef struct { int32_t expert, src, dst, rows; } feplb_move;
+
+/* One segment of the grouped GEMM: rows [row_start, row_start + rows) of the permuted buffers
+ * belong to `expert` and are executed on virtual rank `exec_rank`. */
+typedef struct { int32_t expert, row_start, rows, exec_rank, is_dynamic; } feplb_group;
+
+/* Caller-sized plan.  cap_moves >= R*max_num_dyn and cap_groups >= E + R*max_num_dyn always
+ * suffice; load_before / load_after have R entries.  All host memory, owned by the caller. */
+typedef struct {
+  int32_t n_moves, n_groups;
+  int32_t cap_moves, cap_groups;
+  feplb_move* moves;
+  feplb_group* groups;
+  int64_t* load_before;
+  int64_t* load_after;
+} feplb_plan_out;
+
+/* Host and device timestamps of the last feplb_moe_forward, in microseconds.  Host times count
+ * from the call's entry; device times are CUDA-event intervals on the caller's stream. */
+typedef struct {
+  double host_enqueue_static_done_us; /* host: static-expert GEMM enqueued */
+  double host_counts_ready_us;        /* host planner thread: counts arrived */
+  double host_plan_done_us;           /* host planner thread: plan computed */
+  double host_upload_enqueued_us;     /* host planner thread: group-table upload enqueued */
+  double host_join_us;                /* host: caller joined the planner */
+  double host_return_us;              /* host: everything enqueued */
+  double plan_us;                     /* host: time inside the planner's greedy */
+  double dev_hist_us, dev_dispatch_us, dev_static_ffn_us, dev_dynamic_ffn_us, dev_combine_us;
+  double dev_counts_to_static_start_us; /* device: counts copied -> static GEMM starts */
+  double dev_counts_to_static_end_us;   /* device: counts copied -> static GEMM ends */
+  double dev_total_us;
+} feplb_timeline;
+
+typedef struct feplb_ctx feplb_ctx;
+
+/* ---- library ------------------------------------------------------------------------------ */
+
+/* Version as major*10000 + minor*100 + patch. */
+int feplb_version(void);
+/* Static text for a feplb_status. */
+const char* feplb_strerror(int status);
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Validates `cfg`, selects the current CUDA device, allocates the context's scratch (block
+ * histograms, segment offsets, group tables, pinned staging, status word), creates the copy
+ * stream and starts the planner thread.  *out is NULL on failure. */
+int feplb_create(const feplb_config* cfg, feplb_ctx** out);
+/* Joins the planner thread and frees everything.  NULL is accepted. */
+int feplb_destroy(feplb_ctx* ctx);
+/* Text of the last error recorded on `ctx` (never NULL; empty if none). */
+const char* feplb_last_error(const feplb_ctx* ctx);
+/* Synchronises `stream`, reads and clears the device status word.  Returns FEPLB_OK,
+ * FEPLB_E_RANGE (bad expert id), FEPLB_E_DEVICE (a device-side wait gave up or counts
+ * disagreed with ids) or FEPLB_E_CUDA. */
+int feplb_check_status(feplb_ctx* ctx, void* stream);
+/* Rows the caller must give x_perm, h_scratch, y_perm and row_to_token:
+ * S + E*(A-1), an upper bound of sum_e round_up(counts[e], A); 0 if cfg is invalid. */
+size_t feplb_s_pad(const feplb_config* cfg);
+
+/* ---- host-only steps (no GPU needed) ------------------------------------------------------ */
+
+/* Static/dynamic partition (Section 2.3, parameter dyn): marks the `dyn` highest-scoring
+ * experts of each rank's block in mask_out[E] (host), ties to the lower expert id.  The paper
+ * does not say which experts are dynamic; scoring by this micro-batch's counts is this
+ * library's reading. */
+int feplb_select_dynamic(const int64_t* score, int32_t E, int32_t R, int32_t dyn, uint8_t* mask_out);
+
+/* The greedy load balancer of Section 2.3: repeatedly moves the busiest dynamic expert of the
+ * most loaded rank to the least loaded rank of the same domain, subject to tau, to the receive
+ * capacity max_num_dyn, and to the move lowering the larger of the two loads; deterministic
+ * (ties to the lower rank / expert id).  counts[E] and dyn_mask[E] are host arrays.  Fills
+ * out->moves (ordered), out->groups (expert order; per expert the moved pieces in move order
+ * from the front of its segment, then the home remainder; zero-row groups omitted) and the
+ * per-rank loads.  Returns FEPLB_E_NOMEM if a capacity is too small.  Pure function. */
+int feplb_plan(const feplb_config* cfg, const int32_t* counts, const uint8_t* dyn_mask, feplb_plan_out* out);
+
+/* ---- device steps ------------------------------------------------------------------------- */
+
+/* Step 1 (Section 2.2: per-expert token counts after Phase 1).
+ * topk_ids dev int32 [T,K] -> counts dev int32 [E], rank_load dev int32 [R] (both overwritten).
+ * Ids outside [0,E) are skipped and raise FEPLB_E_RANGE in the status word. */
+int feplb_route_hist(feplb_ctx* ctx, const int32_t* topk_ids, int32_t* counts, int32_t* rank_load, void* stream);
+
+/* Step 3 (Section 2.2: tokens "permuted" for the grouped GEMM) = stable counting sort of the
+ * slots by expert id.  Slot s goes to row pad_off[e] + (earlier slots of e), with
+ * pad_off[e] = sum_{e'<e} round_up(counts[e'], A).
+ *   x dev bf16 [T,d], topk_ids dev [T,K], counts dev [E] (as written by feplb_route_hist)
+ *   -> x_perm dev bf16 [S_cap,d]   (row copies; padding rows inside segments zero-filled)
+ *      slot_to_row dev int32 [T,K], row_to_token dev int32 [S_cap] (-1 where no token). */
+int feplb_dispatch(feplb_ctx* ctx, const void* x, const int32_t* topk_ids, const int32_t* counts,
+                   void* x_perm, int32_t* slot_to_row, int32_t* row_to_token, void* stream);
+
+/* Writes the E-entry group table {e, pad_off[e], counts[e], home(e), dyn_mask[e]} to
+ * groups_out (dev), from device-resident counts and mask, without involving the host: the
+ * table the static-expert GEMM runs on while the planner works (Section 2.3 timeline).
+ * With FEPLB_MASK_REACTIVE pass dyn_mask = NULL: the mask is derived on the device from counts
+ * (same rule as feplb_select_dynamic) and also written to dyn_mask_out (dev uint8 [E], may be NULL). */
+int feplb_home_groups(feplb_ctx* ctx, const int32_t* counts, const uint8_t* dyn_mask,
+                      feplb_group* groups_out, uint8_t* dyn_mask_out, void* stream);
+
+/* Steps 4-5 (Section 2.3: static-expert, then dynamic-expert grouped GEMM).  For every group g
+ * in groups[0..n_groups) selected by `which` (FEPLB_FFN_ALL / _STATIC: is_dynamic == 0 /
+ * _DYNAMIC: is_dynamic != 0) and every row i of it:
+ *   h = silu(x_perm[i] W1[e]) * (x_perm[i] W3[e])   (bf16 x bf16 -> fp32, h rounded to bf16)
+ *   y_perm[i] = h W2[e]                              (fp32 accumulate, rounded to bf16)
+ * Rows outside the selected groups are not written.  groups is a dev array (n_groups <= 1024);
+ * zero-row groups are allowed.  h_scratch dev bf16 [S_cap,f], y_perm dev bf16 [S_cap,d]. */
+int feplb_expert_ffn(feplb_ctx* ctx, const void* x_perm, const void* w1, const void* w3, const void* w2,
+                     const feplb_group* groups, int32_t n_groups, int32_t which,
+                     void* h_scratch, void* y_perm, void* stream);
+
+/* Step 6 (Section 2.3: Combine): out[t,:] = sum_k gates[t,k] * y_perm[slot_to_row[t,k],:],
+ * k ascending, fp32 accumulate, rounded to bf16.  gates dev float [T,K], out dev bf16 [T,d]. */
+int feplb_combine(feplb_ctx* ctx, const void* y_perm, const int32_t* slot_to_row, const float* gates,
+                  void* out, void* stream);
+
+/* ---- planner thread (Section 2.3: CPU balancer on a dedicated thread) ---------------------- */
+
+/* Enqueues on `stream` a copy of counts (dev [E]) to pinned memory and wakes the planner
+ * thread, which waits for the copy (bounded), chooses the mask (dyn_mask_host, host [E], must
+ * stay valid until feplb_plan_wait; NULL with FEPLB_MASK_REACTIVE), runs feplb_plan, and uploads
+ * the dynamic groups on the context's copy stream. */
+int feplb_plan_async(feplb_ctx* ctx, const int32_t* counts, const uint8_t* dyn_mask_host, void* stream);
+/* Waits up to timeout_ms for the planner.  On success copies the plan to *plan_copy (may be
+ * NULL), returns the device table of dynamic groups and its length, and makes `stream` wait
+ * for the upload.  FEPLB_E_TIMEOUT on expiry (the job stays pending), FEPLB_E_STATE if no job. */
+int feplb_plan_wait(feplb_ctx* ctx, int32_t timeout_ms, feplb_plan_out* plan_copy,
+                    const feplb_group** dyn_groups_dev, int32_t* n_dyn_groups, void* stream);
+
+/* ---- whole layer -------------------------------------------------------------------------- */
+
+/* One forward pass of the layer on `stream`: route_hist -> (planner thread || dispatch, static
+ * FFN) -> dynamic FFN -> combine.  Inputs x, topk_ids, gates, w1, w3, w2 (dev).  Outputs and
+ * scratch (dev, caller-owned): counts [E], rank_load [R], x_perm [S_cap,d], h_scratch [S_cap,f],
+ * y_perm [S_cap,d], slot_to_row [T,K], row_to_token [S_cap], out [T,d].  dyn_mask_host: host [E]
+ * or NULL with FEPLB_MASK_REACTIVE.  plan_copy (host, may be NULL) receives the plan.  Blocks the
+ * calling thread only until the planner has enqueued its upload (bounded by 2 s). */
+int feplb_moe_forward(feplb_ctx* ctx, const void* x, const int32_t* topk_ids, const float* gates,
+                      const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                      int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
+                      int32_t* slot_to_row, int32_t* row_to_token, void* out,
+                      feplb_plan_out* plan_copy, void* stream);
+
+/* Same pass with HOST inputs and output: copies x, topk_ids, gates (host, ideally pinned) to
+ * the device buffers x_dev, ids_dev, gates_dev, runs feplb_moe_forward, copies out_dev to
+ * out_host, all on `stream`; returns after the stream has drained.  Weights stay resident. */
+int feplb_moe_forward_host(feplb_ctx* ctx, const void* x_host, const int32_t* topk_ids_host,
+                           const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
+                           const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                           int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
+                           int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
+                           feplb_plan_out* plan_copy, void* stream);
+
+/* Turns CUDA-event timing of the stages of feplb_moe_forward on (1) or off (0, default). */
+int feplb_set_timeline(feplb_ctx* ctx, int32_t enable);
+/* Synchronises the last forward's events and fills *out (device fields are 0 when disabled). */
+int feplb_get_timeline(feplb_ctx* ctx, feplb_timeline* out);
+/* Number of kernels this library has launched on `ctx` since creation. */
+int64_t feplb_launch_count(const feplb_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FEPLB_H_ */

@@ -1,0 +1,519 @@
+// C ABI of libfeplb: context, argument checks, the planner thread (paper Section 2.3: the CPU
+// load balancer runs on a dedicated thread, triggered by router completion, while the GPU
+// computes the static experts) and the per-micro-batch orchestration.
+#include <cuda_runtime.h>
+
+#include <chrono>
+#include <condition_variable>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "feplb.h"
+#include "feplb_internal.h"
+
+namespace {
+using clk = std::chrono::steady_clock;
+inline double us_since(clk::time_point t0) {
+  return std::chrono::duration<double, std::micro>(clk::now() - t0).count();
+}
+enum JobState { JOB_IDLE = 0, JOB_PENDING = 1, JOB_RUNNING = 2, JOB_DONE = 3 };
+enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_N };
+}  // namespace
+
+struct feplb_ctx {
+  feplb_config cfg;
+  int device = 0, num_sms = 0;
+  size_t s_cap = 0;
+  int nb = 0;   // CTAs of the permutation kernels
+  char err[512] = {0};
+  int64_t launches = 0;
+
+  // device scratch
+  int32_t* d_block_hist = nullptr;
+  int32_t* d_pad_off = nullptr;
+  uint32_t* d_status = nullptr;
+  feplb_group* d_home_groups = nullptr;
+  feplb_group* d_dyn_groups = nullptr;
+  uint8_t* d_mask = nullptr;
+  // pinned staging
+  int32_t* h_counts = nullptr;
+  feplb_group* h_dyn_groups = nullptr;
+  uint32_t* h_status = nullptr;
+  uint8_t* h_mask = nullptr;
+
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_counts = nullptr, ev_plan = nullptr;
+  cudaEvent_t ev[EV_N] = {nullptr};
+  bool timeline_on = false, timeline_valid = false;
+  feplb_timeline tl;
+  clk::time_point t0;
+
+  // planner thread
+  std::thread th;
+  std::mutex mu;
+  std::condition_variable cv;
+  bool quit = false;
+  int job = JOB_IDLE;
+  const uint8_t* job_mask = nullptr;
+  int job_rc = FEPLB_OK;
+  int n_dyn_groups = 0;
+  // plan storage owned by the context
+  std::vector<feplb_move> moves;
+  std::vector<feplb_group> groups;
+  std::vector<int64_t> load_before, load_after;
+  std::vector<uint8_t> mask;
+  feplb_plan_out plan;
+};
+
+namespace {
+
+int fail(feplb_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+#define CUDA_TRY(ctx, call)                                                                      \
+  do {                                                                                           \
+    cudaError_t e_ = (call);                                                                     \
+    if (e_ != cudaSuccess) return fail(ctx, FEPLB_E_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// The planner thread: waits for the counts, derives mask and plan, uploads the dynamic groups.
+void planner_main(feplb_ctx* c) {
+  cudaSetDevice(c->device);
+  for (;;) {
+    {
+      std::unique_lock<std::mutex> lk(c->mu);
+      c->cv.wait(lk, [&] { return c->quit || c->job == JOB_PENDING; });
+      if (c->quit) return;
+      c->job = JOB_RUNNING;
+    }
+    int rc = FEPLB_OK;
+    // bounded wait for the copy of the counts (no blocking driver call: poll the event)
+    const auto w0 = clk::now();
+    for (;;) {
+      cudaError_t q = cudaEventQuery(c->ev_counts);
+      if (q == cudaSuccess) break;
+      if (q != cudaErrorNotReady) { rc = FEPLB_E_CUDA; break; }
+      if (std::chrono::duration<double>(clk::now() - w0).count() > 2.0) { rc = FEPLB_E_TIMEOUT; break; }
+    }
+    c->tl.host_counts_ready_us = us_since(c->t0);
+    if (rc == FEPLB_OK) {
+      const feplb_config& cfg = c->cfg;
+      const uint8_t* mask = c->job_mask;
+      if (!mask) {
+        std::vector<int64_t> score(cfg.E);
+        for (int e = 0; e < cfg.E; ++e) score[e] = c->h_counts[e];
+        feplb_select_dynamic(score.data(), cfg.E, cfg.R, cfg.dyn, c->mask.data());
+        mask = c->mask.data();
+      } else {
+        memcpy(c->mask.data(), mask, cfg.E);
+      }
+      const auto p0 = clk::now();
+      rc = feplb_plan(&cfg, c->h_counts, mask, &c->plan);
+      c->tl.plan_us = us_since(p0);
+      c->tl.host_plan_done_us = us_since(c->t0);
+      if (rc == FEPLB_OK) {
+        int n = 0;
+        for (int i = 0; i < c->plan.n_groups; ++i)
+          if (c->plan.groups[i].is_dynamic) c->h_dyn_groups[n++] = c->plan.groups[i];
+        c->n_dyn_groups = n;
+        cudaError_t e = cudaSuccess;
+        if (n) e = cudaMemcpyAsync(c->d_dyn_groups, c->h_dyn_groups, sizeof(feplb_group) * n, cudaMemcpyHostToDevice, c->copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ev_plan, c->copy_stream);
+        if (e != cudaSuccess) rc = FEPLB_E_CUDA;
+      }
+      c->tl.host_upload_enqueued_us = us_since(c->t0);
+    }
+    {
+      std::lock_guard<std::mutex> lk(c->mu);
+      c->job_rc = rc;
+      c->job = JOB_DONE;
+    }
+    c->cv.notify_all();
+  }
+}
+
+int check_dev_ptrs(feplb_ctx* c, std::initializer_list<const void*> ptrs) {
+  for (const void* p : ptrs)
+    if (!p || !aligned16(p)) return fail(c, FEPLB_E_INVALID, "null or unaligned device pointer");
+  return FEPLB_OK;
+}
+
+}  // namespace
+
+extern "C" int feplb_version(void) { return 100; }
+
+extern "C" const char* feplb_strerror(int s) {
+  switch (s) {
+    case FEPLB_OK: return "ok";
+    case FEPLB_E_INVALID: return "invalid argument";
+    case FEPLB_E_RANGE: return "expert id out of range";
+    case FEPLB_E_CUDA: return "CUDA error";
+    case FEPLB_E_NOMEM: return "out of memory or capacity too small";
+    case FEPLB_E_TIMEOUT: return "timed out";
+    case FEPLB_E_STATE: return "invalid call order";
+    case FEPLB_E_DEVICE: return "device-side check failed";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
+  if (!out) return FEPLB_E_INVALID;
+  *out = nullptr;
+  int rc = feplb_validate_config(cfg);
+  if (rc != FEPLB_OK) return rc;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FEPLB_E_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return FEPLB_E_CUDA;
+  if (prop.major != 10) return FEPLB_E_CUDA;   // sm_100a code only
+  feplb_ctx* c = new (std::nothrow) feplb_ctx();
+  if (!c) return FEPLB_E_NOMEM;
+  c->cfg = *cfg;
+  c->device = dev;
+  c->num_sms = prop.multiProcessorCount;
+  c->s_cap = feplb_s_pad(cfg);
+  const int64_t S = (int64_t)cfg->T * cfg->K;
+  c->nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
+  const int cap_moves = cfg->R * cfg->max_num_dyn;
+  const int cap_groups = cfg->E + cap_moves;
+  bool ok = true;
+  ok = ok && cudaMalloc(&c->d_block_hist, sizeof(int32_t) * (size_t)(c->nb > 0 ? c->nb : 1) * cfg->E) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_pad_off, sizeof(int32_t) * (cfg->E + 1)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_status, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_home_groups, sizeof(feplb_group) * cfg->E) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_mask, cfg->E) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_counts, sizeof(int32_t) * cfg->E) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_status, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_mask, cfg->E) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreate(&c->ev_counts) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < EV_N; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    feplb_destroy(c);
+    return FEPLB_E_NOMEM;
+  }
+  c->moves.resize(cap_moves > 0 ? cap_moves : 1);
+  c->groups.resize(cap_groups);
+  c->load_before.resize(cfg->R);
+  c->load_after.resize(cfg->R);
+  c->mask.resize(cfg->E);
+  c->plan = feplb_plan_out{0, 0, cap_moves, cap_groups, c->moves.data(), c->groups.data(),
+                           c->load_before.data(), c->load_after.data()};
+  memset(&c->tl, 0, sizeof(c->tl));
+  c->th = std::thread(planner_main, c);
+  *out = c;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_destroy(feplb_ctx* c) {
+  if (!c) return FEPLB_OK;
+  if (c->th.joinable()) {
+    {
+      std::lock_guard<std::mutex> lk(c->mu);
+      c->quit = true;
+    }
+    c->cv.notify_all();
+    c->th.join();
+  }
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  cudaFree(c->d_block_hist);
+  cudaFree(c->d_pad_off);
+  cudaFree(c->d_status);
+  cudaFree(c->d_home_groups);
+  cudaFree(c->d_dyn_groups);
+  cudaFree(c->d_mask);
+  cudaFreeHost(c->h_counts);
+  cudaFreeHost(c->h_dyn_groups);
+  cudaFreeHost(c->h_status);
+  cudaFreeHost(c->h_mask);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->ev_counts) cudaEventDestroy(c->ev_counts);
+  if (c->ev_plan) cudaEventDestroy(c->ev_plan);
+  for (int i = 0; i < EV_N; ++i)
+    if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  cudaGetLastError();
+  delete c;
+  return FEPLB_OK;
+}
+
+extern "C" const char* feplb_last_error(const feplb_ctx* c) { return c ? c->err : ""; }
+
+extern "C" int64_t feplb_launch_count(const feplb_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int feplb_check_status(feplb_ctx* c, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaMemsetAsync(c->d_status, 0, sizeof(uint32_t), st));
+  CUDA_TRY(c, cudaStreamSynchronize(st));
+  const uint32_t s = *c->h_status;
+  if (s & FEPLB_ST_WAIT) return fail(c, FEPLB_E_DEVICE, "a bounded device-side wait gave up (status 0x%x)", s);
+  if (s & FEPLB_ST_GROUP) return fail(c, FEPLB_E_DEVICE, "malformed group entry (status 0x%x)", s);
+  if (s & FEPLB_ST_COUNTS) return fail(c, FEPLB_E_DEVICE, "counts disagree with topk_ids (status 0x%x)", s);
+  if (s & FEPLB_ST_RANGE) return fail(c, FEPLB_E_RANGE, "expert id outside [0, E) (status 0x%x)", s);
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_route_hist(feplb_ctx* c, const int32_t* topk_ids, int32_t* counts, int32_t* rank_load, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (!counts || !rank_load || (!topk_ids && c->cfg.T > 0)) return fail(c, FEPLB_E_INVALID, "route_hist: null pointer");
+  const int64_t S = (int64_t)c->cfg.T * c->cfg.K;
+  CUDA_TRY(c, feplb_launch_block_hist(topk_ids, S, c->cfg.E, c->cfg.R, c->d_block_hist, counts, rank_load,
+                                      c->d_status, (cudaStream_t)stream, &c->launches));
+  return FEPLB_OK;
+}
+
+static int dispatch_impl(feplb_ctx* c, const void* x, const int32_t* topk_ids, const int32_t* counts, void* x_perm,
+                         int32_t* slot_to_row, int32_t* row_to_token, cudaStream_t st) {
+  const feplb_config& g = c->cfg;
+  const int64_t S = (int64_t)g.T * g.K;
+  if (!counts || !row_to_token) return fail(c, FEPLB_E_INVALID, "dispatch: null pointer");
+  if (g.T > 0) {
+    int rc = check_dev_ptrs(c, {x, x_perm});
+    if (rc != FEPLB_OK) return rc;
+    if (!topk_ids || !slot_to_row) return fail(c, FEPLB_E_INVALID, "dispatch: null pointer");
+  }
+  CUDA_TRY(c, feplb_launch_permute(topk_ids, S, g.K, g.E, g.row_align, counts, c->d_block_hist, c->d_pad_off,
+                                   slot_to_row, row_to_token, (int64_t)c->s_cap, c->d_status, st, &c->launches));
+  CUDA_TRY(c, feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
+                                  st, &c->launches));
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_dispatch(feplb_ctx* c, const void* x, const int32_t* topk_ids, const int32_t* counts,
+                              void* x_perm, int32_t* slot_to_row, int32_t* row_to_token, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  return dispatch_impl(c, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, (cudaStream_t)stream);
+}
+
+extern "C" int feplb_home_groups(feplb_ctx* c, const int32_t* counts, const uint8_t* dyn_mask,
+                                 feplb_group* groups_out, uint8_t* dyn_mask_out, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (!counts || !groups_out) return fail(c, FEPLB_E_INVALID, "home_groups: null pointer");
+  if (!dyn_mask && c->cfg.mask_policy != FEPLB_MASK_REACTIVE)
+    return fail(c, FEPLB_E_INVALID, "home_groups: dyn_mask is required unless mask_policy is REACTIVE");
+  CUDA_TRY(c, feplb_launch_home_groups(counts, dyn_mask, c->cfg.E, c->cfg.R, c->cfg.row_align, c->cfg.dyn,
+                                       groups_out, dyn_mask_out, (cudaStream_t)stream, &c->launches));
+  return FEPLB_OK;
+}
+
+static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void* w3, const void* w2,
+                    const feplb_group* groups, int32_t n_groups, int32_t which, void* h, void* y, cudaStream_t st) {
+  if (n_groups < 0 || n_groups > FEPLB_MAX_GROUPS) return fail(c, FEPLB_E_INVALID, "expert_ffn: n_groups out of range");
+  if (which != FEPLB_FFN_ALL && which != FEPLB_FFN_STATIC && which != FEPLB_FFN_DYNAMIC)
+    return fail(c, FEPLB_E_INVALID, "expert_ffn: bad selector");
+  if (n_groups == 0 || c->s_cap == 0) return FEPLB_OK;
+  int rc = check_dev_ptrs(c, {x_perm, w1, w3, w2, h, y});
+  if (rc != FEPLB_OK) return rc;
+  if (!groups) return fail(c, FEPLB_E_INVALID, "expert_ffn: null group table");
+  feplb_gemm_args a;
+  a.x_perm = x_perm; a.w1 = w1; a.w3 = w3; a.w2 = w2; a.h = h; a.y = y;
+  a.groups = groups; a.n_groups = n_groups; a.which = which;
+  a.E = c->cfg.E; a.d = c->cfg.d; a.f = c->cfg.f; a.s_cap = (int64_t)c->s_cap;
+  a.status = c->d_status; a.num_sms = c->num_sms;
+  return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err));
+}
+
+extern "C" int feplb_expert_ffn(feplb_ctx* c, const void* x_perm, const void* w1, const void* w3, const void* w2,
+                                const feplb_group* groups, int32_t n_groups, int32_t which,
+                                void* h_scratch, void* y_perm, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  return ffn_impl(c, x_perm, w1, w3, w2, groups, n_groups, which, h_scratch, y_perm, (cudaStream_t)stream);
+}
+
+extern "C" int feplb_combine(feplb_ctx* c, const void* y_perm, const int32_t* slot_to_row, const float* gates,
+                             void* out, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (c->cfg.T == 0) return FEPLB_OK;
+  int rc = check_dev_ptrs(c, {y_perm, out});
+  if (rc != FEPLB_OK) return rc;
+  if (!slot_to_row || !gates) return fail(c, FEPLB_E_INVALID, "combine: null pointer");
+  CUDA_TRY(c, feplb_launch_combine(y_perm, slot_to_row, gates, out, c->cfg.T, c->cfg.K, c->cfg.d,
+                                   (cudaStream_t)stream, &c->launches));
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_plan_async(feplb_ctx* c, const int32_t* counts, const uint8_t* dyn_mask_host, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (!counts) return fail(c, FEPLB_E_INVALID, "plan_async: null counts");
+  if (!dyn_mask_host && c->cfg.mask_policy != FEPLB_MASK_REACTIVE)
+    return fail(c, FEPLB_E_INVALID, "plan_async: dyn_mask_host is required unless mask_policy is REACTIVE");
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "plan_async: a plan is already pending");
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!c->timeline_valid) c->t0 = clk::now();
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_counts, counts, sizeof(int32_t) * c->cfg.E, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaEventRecord(c->ev_counts, st));
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    c->job_mask = dyn_mask_host;
+    c->job = JOB_PENDING;
+  }
+  c->cv.notify_all();
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out* plan_copy,
+                               const feplb_group** dyn_groups_dev, int32_t* n_dyn_groups, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  int rc;
+  {
+    std::unique_lock<std::mutex> lk(c->mu);
+    if (c->job == JOB_IDLE) return fail(c, FEPLB_E_STATE, "plan_wait: no plan was requested");
+    if (!c->cv.wait_for(lk, std::chrono::milliseconds(timeout_ms < 0 ? 0 : timeout_ms), [&] { return c->job == JOB_DONE; }))
+      return fail(c, FEPLB_E_TIMEOUT, "plan_wait: planner did not finish within %d ms", timeout_ms);
+    rc = c->job_rc;
+    c->job = JOB_IDLE;
+  }
+  if (rc != FEPLB_OK) return fail(c, rc, "planner failed: %s", feplb_strerror(rc));
+  if (plan_copy) {
+    if (plan_copy->cap_moves < c->plan.n_moves || plan_copy->cap_groups < c->plan.n_groups ||
+        !plan_copy->load_before || !plan_copy->load_after)
+      return fail(c, FEPLB_E_NOMEM, "plan_wait: plan_copy too small");
+    plan_copy->n_moves = c->plan.n_moves;
+    plan_copy->n_groups = c->plan.n_groups;
+    if (c->plan.n_moves) memcpy(plan_copy->moves, c->plan.moves, sizeof(feplb_move) * c->plan.n_moves);
+    if (c->plan.n_groups) memcpy(plan_copy->groups, c->plan.groups, sizeof(feplb_group) * c->plan.n_groups);
+    memcpy(plan_copy->load_before, c->plan.load_before, sizeof(int64_t) * c->cfg.R);
+    memcpy(plan_copy->load_after, c->plan.load_after, sizeof(int64_t) * c->cfg.R);
+  }
+  if (dyn_groups_dev) *dyn_groups_dev = c->d_dyn_groups;
+  if (n_dyn_groups) *n_dyn_groups = c->n_dyn_groups;
+  CUDA_TRY(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_plan, 0));
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_set_timeline(feplb_ctx* c, int32_t enable) {
+  if (!c) return FEPLB_E_INVALID;
+  c->timeline_on = enable != 0;
+  return FEPLB_OK;
+}
+
+#define TL_EVENT(i)                                                  \
+  do {                                                               \
+    if (c->timeline_on) CUDA_TRY(c, cudaEventRecord(c->ev[i], st));  \
+  } while (0)
+
+extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* topk_ids, const float* gates,
+                                 const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                                 int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
+                                 int32_t* slot_to_row, int32_t* row_to_token, void* out,
+                                 feplb_plan_out* plan_copy, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  const feplb_config& g = c->cfg;
+  if (!dyn_mask_host && g.mask_policy != FEPLB_MASK_REACTIVE)
+    return fail(c, FEPLB_E_INVALID, "moe_forward: dyn_mask_host is required unless mask_policy is REACTIVE");
+  c->t0 = clk::now();
+  c->timeline_valid = true;
+  int rc;
+  TL_EVENT(EV_T0);
+  // step 1: counts; the planner thread starts as soon as they reach the host
+  if ((rc = feplb_route_hist(c, topk_ids, counts, rank_load, stream)) != FEPLB_OK) return rc;
+  if ((rc = feplb_plan_async(c, counts, dyn_mask_host, stream)) != FEPLB_OK) return rc;
+  TL_EVENT(EV_HIST);
+  // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move them here)
+  rc = dispatch_impl(c, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, st);
+  TL_EVENT(EV_DISPATCH);
+  // step 4: static experts on their home ranks, from a group table built on the device
+  if (rc == FEPLB_OK) {
+    const uint8_t* mask_dev = nullptr;
+    if (dyn_mask_host) {
+      memcpy(c->h_mask, dyn_mask_host, g.E);
+      cudaError_t e = cudaMemcpyAsync(c->d_mask, c->h_mask, g.E, cudaMemcpyHostToDevice, st);
+      if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "mask upload: %s", cudaGetErrorString(e));
+      mask_dev = c->d_mask;
+    }
+    if (rc == FEPLB_OK) rc = feplb_home_groups(c, counts, mask_dev, c->d_home_groups, nullptr, stream);
+  }
+  TL_EVENT(EV_STATIC0);
+  if (rc == FEPLB_OK)
+    rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st);
+  TL_EVENT(EV_STATIC1);
+  c->tl.host_enqueue_static_done_us = us_since(c->t0);
+  // join the planner (always, so that the context returns to idle), then step 5
+  const feplb_group* dyn_groups = nullptr;
+  int32_t n_dyn = 0;
+  int rc_join = feplb_plan_wait(c, 2000, plan_copy, &dyn_groups, &n_dyn, stream);
+  c->tl.host_join_us = us_since(c->t0);
+  if (rc != FEPLB_OK) return rc;
+  if (rc_join != FEPLB_OK) return rc_join;
+  TL_EVENT(EV_DYN0);
+  if ((rc = ffn_impl(c, x_perm, w1, w3, w2, dyn_groups, n_dyn, FEPLB_FFN_ALL, h_scratch, y_perm, st)) != FEPLB_OK) return rc;
+  TL_EVENT(EV_DYN1);
+  // step 6
+  if ((rc = feplb_combine(c, y_perm, slot_to_row, gates, out, stream)) != FEPLB_OK) return rc;
+  TL_EVENT(EV_COMBINE);
+  c->tl.host_return_us = us_since(c->t0);
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_moe_forward_host(feplb_ctx* c, const void* x_host, const int32_t* topk_ids_host,
+                                      const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
+                                      const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                                      int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
+                                      int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
+                                      feplb_plan_out* plan_copy, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  const feplb_config& g = c->cfg;
+  const size_t nx = (size_t)g.T * g.d * 2, nk = (size_t)g.T * g.K * 4;
+  if (g.T > 0) {
+    if (!x_host || !topk_ids_host || !gates_host || !out_host || !x_dev || !ids_dev || !gates_dev || !out_dev)
+      return fail(c, FEPLB_E_INVALID, "moe_forward_host: null pointer");
+    CUDA_TRY(c, cudaMemcpyAsync(ids_dev, topk_ids_host, nk, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(c, cudaMemcpyAsync(gates_dev, gates_host, nk, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(c, cudaMemcpyAsync(x_dev, x_host, nx, cudaMemcpyHostToDevice, st));
+  }
+  int rc = feplb_moe_forward(c, x_dev, ids_dev, gates_dev, w1, w3, w2, dyn_mask_host, counts, rank_load, x_perm,
+                             h_scratch, y_perm, slot_to_row, row_to_token, out_dev, plan_copy, stream);
+  if (rc != FEPLB_OK) return rc;
+  if (g.T > 0) CUDA_TRY(c, cudaMemcpyAsync(out_host, out_dev, nx, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaStreamSynchronize(st));
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_get_timeline(feplb_ctx* c, feplb_timeline* out) {
+  if (!c || !out) return FEPLB_E_INVALID;
+  if (!c->timeline_valid) return fail(c, FEPLB_E_STATE, "get_timeline: no forward pass yet");
+  feplb_timeline t = c->tl;
+  t.dev_hist_us = t.dev_dispatch_us = t.dev_static_ffn_us = t.dev_dynamic_ffn_us = t.dev_combine_us = 0;
+  t.dev_counts_to_static_start_us = t.dev_counts_to_static_end_us = t.dev_total_us = 0;
+  if (c->timeline_on) {
+    CUDA_TRY(c, cudaEventSynchronize(c->ev[EV_COMBINE]));
+    float ms = 0;
+    auto el = [&](cudaEvent_t a, cudaEvent_t b) { return cudaEventElapsedTime(&ms, a, b) == cudaSuccess ? ms * 1e3 : 0.0; };
+    t.dev_hist_us = el(c->ev[EV_T0], c->ev[EV_HIST]);
+    t.dev_dispatch_us = el(c->ev[EV_HIST], c->ev[EV_DISPATCH]);
+    t.dev_static_ffn_us = el(c->ev[EV_STATIC0], c->ev[EV_STATIC1]);
+    t.dev_dynamic_ffn_us = el(c->ev[EV_DYN0], c->ev[EV_DYN1]);
+    t.dev_combine_us = el(c->ev[EV_DYN1], c->ev[EV_COMBINE]);
+    t.dev_counts_to_static_start_us = el(c->ev_counts, c->ev[EV_STATIC0]);
+    t.dev_counts_to_static_end_us = el(c->ev_counts, c->ev[EV_STATIC1]);
+    t.dev_total_us = el(c->ev[EV_T0], c->ev[EV_COMBINE]);
+    cudaGetLastError();
+  }
+  *out = t;
+  return FEPLB_OK;
+}

@@ -1,0 +1,482 @@
+// Grouped SwiGLU expert FFN of the FEPLB hot path on sm_100a (paper Section 2.3: static-expert,
+// then dynamic-expert Grouped GEMM; Section 3.1: grouped GEMM over per-expert row segments).
+//
+// Two launches of one persistent, warp-specialised kernel:
+//   pass 1 (SwiGLU): H[rows, n0:n0+bn] = silu(X W1[e]) * (X W3[e])   -- one MMA of N = 2*bn whose
+//                    B tile is the W1 tile followed by the W3 tile; the epilogue multiplies
+//                    the two halves of the accumulator and rounds to bf16
+//   pass 2 (plain):  Y[rows, n0:n0+2bn] = H W2[e]
+// Per CTA: warp 0 = TMA producer (one lane), warp 1 = tcgen05.mma issuer (one lane) and TMEM
+// owner, warps 2..5 = epilogue (tcgen05.ld -> registers -> global).  A and B tiles are staged
+// by TMA (128-byte swizzle, K-major) through a 4-stage shared-memory ring; the fp32 accumulator
+// lives in TMEM and is double-buffered so the epilogue of tile i overlaps the MMAs of tile
+// i+1.  A tile is 128 rows of ONE group (row segment of one expert); the last tile of a group
+// is ragged and its surplus rows are computed but never stored.
+//
+// Every mbarrier wait is bounded: when it gives up the CTA raises FEPLB_ST_WAIT in the status
+// word, all roles leave their loops, TMEM is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+
+#include "feplb_internal.h"
+
+namespace {
+
+constexpr int BM = FEPLB_TILE_M;       // rows per tile (UMMA M)
+constexpr int BK = 64;                 // K elements per stage = one 128-byte swizzle row
+constexpr int UMMA_K = 16;             // K per tcgen05.mma for 16-bit inputs
+constexpr int kStages = 4;
+constexpr int kAccStages = 2;
+constexpr int kAccCols = 256;          // TMEM columns per accumulator stage
+constexpr int kTmemCols = kAccStages * kAccCols;   // 512 = all of TMEM: one CTA per SM
+constexpr int kThreads = 192;
+constexpr int kABytes = BM * BK * 2;               // 16 KiB
+constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytesMax;  // 48 KiB, a multiple of 1024
+constexpr unsigned long long kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s per wait
+
+struct SmemTail {
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long tmem_full[kAccStages];
+  unsigned long long tmem_empty[kAccStages];
+  uint32_t tmem_base;
+  int abort_flag;
+  int prefix[FEPLB_MAX_GROUPS + 1];   // prefix[g] = M-tiles of groups before g
+  int g_row_start[FEPLB_MAX_GROUPS];
+  int g_rows[FEPLB_MAX_GROUPS];
+  int g_expert[FEPLB_MAX_GROUPS];
+};
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(SmemTail);
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+static_assert(kSmemBytes > 116 * 1024, "two CTAs must never share an SM: each allocates all of TMEM");
+
+struct GemmParams {
+  const feplb_group* groups;
+  int n_groups;
+  int which;            // FEPLB_FFN_*
+  int E;
+  int64_t s_cap;        // rows of the A and output buffers
+  int n_tiles_n;        // N tiles per M tile
+  int num_k_blocks;     // K / 64
+  int b_rows_per_expert;  // rows of one expert in the B tensor maps
+  int bn;               // rows of one B half tile (64 or 128); the MMA has N = 2*bn
+  int swiglu;           // 1: out = silu(acc[:bn]) * acc[bn:], bn columns; 0: out = acc, 2*bn columns
+  __nv_bfloat16* out;
+  int ld_out;           // elements between output rows
+  uint32_t* status;
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the limit expired.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicOr(status, FEPLB_ST_WAIT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+
+// 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier of this CTA.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate, issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival once all tcgen05.mma issued so far by this thread are done.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns of TMEM -> 32 registers per thread (thread i = lane i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) wide and
+// 128-byte swizzled, 8-row groups 1024 bytes apart: start address >> 4 in bits [0,14), leading
+// byte offset (unused for swizzled K-major) = 1 in [16,30), stride byte offset 1024 >> 4 in
+// [32,46), descriptor version 1 in [46,48), layout type 2 (SWIZZLE_128B) in [61,64).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor of tcgen05.mma kind::f16: D fp32 (bits [4,6) = 1), A and B bf16
+// ([7,10) = 1, [10,13) = 1), both K-major (bits 15, 16 = 0), N >> 3 in [17,23), M >> 4 in [24,29).
+__device__ __forceinline__ uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float silu_f(float a) { return __fdividef(a, 1.f + __expf(-a)); }
+
+struct TileCoord { int row0, rows_valid, expert, nt; };
+
+// tile -> (group, M tile, N tile); N tiles of one M tile are consecutive so that CTAs running at
+// the same time share the A rows and sweep one expert's weights together (both stay in L2).
+__device__ __forceinline__ TileCoord tile_coord(const SmemTail* t, int n_groups, int n_tiles_n, int tile) {
+  const int mt = tile / n_tiles_n;
+  int lo = 0, hi = n_groups;   // largest g with prefix[g] <= mt
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t->prefix[mid] <= mt) lo = mid; else hi = mid;
+  }
+  const int local = mt - t->prefix[lo];
+  TileCoord c;
+  c.row0 = t->g_row_start[lo] + local * BM;
+  c.rows_valid = min(BM, t->g_rows[lo] - local * BM);
+  c.expert = t->g_expert[lo];
+  c.nt = tile - mt * n_tiles_n;
+  return c;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+               const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  SmemTail* tail = reinterpret_cast<SmemTail*>(smem + (size_t)kStages * kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &tail->abort_flag;
+
+  // ---- set-up: barriers, TMEM, group table ------------------------------------------------
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_b0);
+    prefetch_tmap(&tm_b1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&tail->full[s]), 1);
+      mbar_init(smem_u32(&tail->empty[s]), 1);
+    }
+    for (int a = 0; a < kAccStages; ++a) {
+      mbar_init(smem_u32(&tail->tmem_full[a]), 1);
+      mbar_init(smem_u32(&tail->tmem_empty[a]), 4);   // one arrival per epilogue warp
+    }
+    tail->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  for (int g = threadIdx.x; g < p.n_groups; g += kThreads) {
+    const feplb_group gr = p.groups[g];
+    const bool selected = p.which == FEPLB_FFN_ALL || (p.which == FEPLB_FFN_STATIC) == (gr.is_dynamic == 0);
+    int tiles = 0;
+    if (selected && gr.rows > 0) {
+      const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 &&
+                      (int64_t)gr.row_start + gr.rows <= p.s_cap;
+      if (ok) tiles = (gr.rows + BM - 1) / BM;
+      else atomicOr(p.status, FEPLB_ST_GROUP);
+    }
+    tail->prefix[g + 1] = tiles;   // turned into a prefix sum below
+    tail->g_row_start[g] = gr.row_start;
+    tail->g_rows[g] = gr.rows;
+    tail->g_expert[g] = gr.expert;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    // exclusive scan of the per-group tile counts, 32 lanes x contiguous chunks
+    const int per = (p.n_groups + 31) / 32;
+    const int g0 = lane * per, g1 = min(p.n_groups, g0 + per);
+    int sum = 0;
+    for (int g = g0; g < g1; ++g) sum += tail->prefix[g + 1];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    int run = incl - sum;
+    for (int g = g0; g < g1; ++g) {
+      const int t = tail->prefix[g + 1];
+      run += t;
+      tail->prefix[g + 1] = run;
+    }
+    if (lane == 0) tail->prefix[0] = 0;
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  const int total_tiles = tail->prefix[p.n_groups] * p.n_tiles_n;
+  const uint32_t b_half_bytes = (uint32_t)p.bn * BK * 2;
+  const uint32_t stage_tx = kABytes + 2 * b_half_bytes;
+
+  if (warp == 0) {
+    // ---- TMA producer ---------------------------------------------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const TileCoord c = tile_coord(tail, p.n_groups, p.n_tiles_n, tile);
+        const int brow0 = c.expert * p.b_rows_per_expert + (p.swiglu ? c.nt * p.bn : c.nt * 2 * p.bn);
+        const int brow1 = p.swiglu ? brow0 : brow0 + p.bn;
+        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+          if (!(ok = mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status))) break;
+          const uint32_t full = smem_u32(&tail->full[stage]);
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
+          const uint32_t sb = sa + kABytes;
+          mbar_expect_tx(full, stage_tx);
+          tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
+          tma_load_2d(sb, &tm_b0, full, kb * BK, brow0);
+          tma_load_2d(sb + b_half_bytes, &tm_b1, full, kb * BK, brow1);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // leave time for copies already issued to land before the CTA's shared memory goes away
+        for (int i = 0; i < 2000; ++i) __nanosleep(100);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer -------------------------------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(BM, 2 * p.bn);
+      int stage = 0, as = 0;
+      uint32_t phase = 0, aphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        if (!(ok = mbar_wait(smem_u32(&tail->tmem_empty[as]), aphase ^ 1u, abort_flag, p.status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(as * kAccCols);
+        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+          if (!(ok = mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // +32 bytes (>> 4 = 2) per K step inside the 128-byte swizzle row
+            umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+          }
+          umma_commit(smem_u32(&tail->empty[stage]));   // stage reusable once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&tail->tmem_full[as]));     // accumulator complete
+        if (++as == kAccStages) { as = 0; aphase ^= 1u; }
+      }
+    }
+  } else {
+    // ---- epilogue: TMEM -> registers -> global ----------------------------------------------
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int row_local = q * 32 + lane;
+    int as = 0;
+    uint32_t aphase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const TileCoord c = tile_coord(tail, p.n_groups, p.n_tiles_n, tile);
+      ok = mbar_wait(smem_u32(&tail->tmem_full[as]), aphase, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * kAccCols);
+      const bool valid = row_local < c.rows_valid;
+      const int out_cols = p.swiglu ? p.bn : 2 * p.bn;
+      __nv_bfloat16* orow = p.out + (int64_t)(c.row0 + row_local) * p.ld_out + (int64_t)c.nt * out_cols;
+      for (int col = 0; col < out_cols; col += 32) {
+        uint32_t a[32];
+        uint32_t packed[16];
+        tmem_ld32(taddr + (uint32_t)col, a);
+        if (p.swiglu) {
+          uint32_t b[32];
+          tmem_ld32(taddr + (uint32_t)(p.bn + col), b);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float h0 = silu_f(__uint_as_float(a[2 * i])) * __uint_as_float(b[2 * i]);
+            const float h1 = silu_f(__uint_as_float(a[2 * i + 1])) * __uint_as_float(b[2 * i + 1]);
+            packed[i] = pack_bf16x2(h0, h1);
+          }
+        } else {
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            packed[i] = pack_bf16x2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+        }
+        if (valid) {
+          uint4* dst = reinterpret_cast<uint4*>(orow + col);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      if (++as == kAccStages) { as = 0; aphase ^= 1u; }
+    }
+  }
+
+  // ---- teardown ---------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_fn() {
+  static encode_tiled_fn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_tiled_fn>(p);
+  }
+  return fn;
+}
+
+// Row-major bf16 matrix [rows, inner] -> tensor map with a [box_rows, 64] box, 128-byte swizzle.
+bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn) {
+  if (a.n_groups == 0 || a.s_cap == 0) return FEPLB_OK;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_grouped_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) {
+      snprintf(err, errn, "cudaFuncSetAttribute(k_grouped_gemm): %s", cudaGetErrorString(e));
+      return FEPLB_E_CUDA;
+    }
+    attr_set = true;
+  }
+  // pass 1: H = silu(X W1) * (X W3);  N tile = bn columns of H, MMA N = 2*bn
+  const int bn1 = (a.f % 128 == 0) ? 128 : 64;
+  // pass 2: Y = H W2;  N tile = 2*bn columns of Y
+  const int bn2 = (a.d % 256 == 0) ? 128 : 64;
+  CUtensorMap tm_x, tm_w1, tm_w3, tm_h, tm_w2;
+  if (!make_tmap(&tm_x, a.x_perm, (uint64_t)a.s_cap, (uint64_t)a.d, BM) ||
+      !make_tmap(&tm_w1, a.w1, (uint64_t)a.E * a.f, (uint64_t)a.d, bn1) ||
+      !make_tmap(&tm_w3, a.w3, (uint64_t)a.E * a.f, (uint64_t)a.d, bn1) ||
+      !make_tmap(&tm_h, a.h, (uint64_t)a.s_cap, (uint64_t)a.f, BM) ||
+      !make_tmap(&tm_w2, a.w2, (uint64_t)a.E * a.d, (uint64_t)a.f, bn2)) {
+    snprintf(err, errn, "cuTensorMapEncodeTiled failed (driver entry point missing or bad pointer/shape)");
+    return FEPLB_E_CUDA;
+  }
+  GemmParams p1;
+  p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
+  p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1; p1.swiglu = 1;
+  p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status;
+  GemmParams p2 = p1;
+  p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2; p2.swiglu = 0;
+  p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d;
+
+  k_grouped_gemm<<<a.num_sms, kThreads, kSmemBytes, st>>>(tm_x, tm_w1, tm_w3, p1);
+  ++*n_launch;
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) {
+    k_grouped_gemm<<<a.num_sms, kThreads, kSmemBytes, st>>>(tm_h, tm_w2, tm_w2, p2);
+    ++*n_launch;
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    snprintf(err, errn, "k_grouped_gemm launch: %s", cudaGetErrorString(e));
+    return FEPLB_E_CUDA;
+  }
+  return FEPLB_OK;
+}

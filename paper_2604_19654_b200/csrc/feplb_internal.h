@@ -1,0 +1,55 @@
+// Internal declarations shared by the translation units of libfeplb (not part of the ABI).
+#ifndef FEPLB_INTERNAL_H_
+#define FEPLB_INTERNAL_H_
+
+#include <cstddef>
+#include <cstdint>
+
+#include "feplb.h"
+
+#define FEPLB_MAX_EXPERTS 1024
+#define FEPLB_MAX_GROUPS 1024
+#define FEPLB_SLOTS_PER_BLOCK 1024   // slots ranked by one CTA of the permutation kernels
+#define FEPLB_TILE_M 128             // rows of one GEMM tile
+
+// bits of the device status word
+#define FEPLB_ST_RANGE 1u      // expert id outside [0, E)
+#define FEPLB_ST_COUNTS 2u     // counts passed to dispatch disagree with the ids
+#define FEPLB_ST_WAIT 4u       // a bounded mbarrier wait gave up inside the GEMM
+#define FEPLB_ST_GROUP 8u      // a group entry was malformed (expert or rows out of range)
+
+int feplb_validate_config(const feplb_config* c);
+
+#ifdef __CUDACC__
+#include <cuda_runtime.h>
+
+// Kernel launchers (each enqueues on `st` and returns the cudaError_t of the launch).
+// n_launch is incremented by the number of kernels enqueued.
+cudaError_t feplb_launch_block_hist(const int32_t* ids, int64_t S, int E, int R, int32_t* block_hist,
+                                    int32_t* counts, int32_t* rank_load, uint32_t* status,
+                                    cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, int A, const int32_t* counts,
+                                 int32_t* block_hist, int32_t* pad_off, int32_t* slot_to_row,
+                                 int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                 cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
+                                const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
+                                cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
+                                     feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row, const float* gates, void* out,
+                                 int T, int K, int d, cudaStream_t st, int64_t* n_launch);
+
+struct feplb_gemm_args {
+  const void* x_perm; const void* w1; const void* w3; const void* w2;
+  void* h; void* y;
+  const feplb_group* groups; int n_groups; int which;
+  int E, d, f; int64_t s_cap;
+  uint32_t* status;
+  int num_sms;
+};
+// Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
+int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
+#endif
+
+#endif  // FEPLB_INTERNAL_H_

@@ -1,0 +1,140 @@
+// Host-side steps of the FEPLB hot path: the static/dynamic partition and the greedy
+// per-micro-batch load balancer (paper Section 2.3).  Pure C++, no CUDA: the planner thread of
+// the library and callers without a GPU run exactly this code.
+#include <algorithm>
+#include <cstdint>
+#include <vector>
+
+#include "feplb.h"
+#include "feplb_internal.h"
+
+int feplb_validate_config(const feplb_config* c) {
+  if (!c) return FEPLB_E_INVALID;
+  if (c->T < 0 || c->K < 1 || c->K > 32 || c->E < 1 || c->E > FEPLB_MAX_EXPERTS || c->R < 1) return FEPLB_E_INVALID;
+  if (c->E % c->R) return FEPLB_E_INVALID;
+  if (c->d < 128 || c->d % 128 || c->f < 64 || c->f % 64) return FEPLB_E_INVALID;
+  if (c->row_align != 1 && c->row_align != 128) return FEPLB_E_INVALID;
+  if (c->split_granule < 1 || c->max_num_dyn < 0 || c->tau < 0 || c->dyn < 0) return FEPLB_E_INVALID;
+  if (c->ranks_per_domain < 0 || (c->ranks_per_domain > 0 && c->R % c->ranks_per_domain)) return FEPLB_E_INVALID;
+  if (c->policy != FEPLB_POLICY_LITERAL && c->policy != FEPLB_POLICY_FIRST_FIT) return FEPLB_E_INVALID;
+  if (c->split != 0 && c->split != 1) return FEPLB_E_INVALID;
+  if (c->mask_policy != FEPLB_MASK_GIVEN && c->mask_policy != FEPLB_MASK_REACTIVE) return FEPLB_E_INVALID;
+  if ((int64_t)c->T * c->K + (int64_t)c->E * (c->row_align - 1) > INT32_MAX) return FEPLB_E_INVALID;
+  return FEPLB_OK;
+}
+
+extern "C" size_t feplb_s_pad(const feplb_config* c) {
+  if (feplb_validate_config(c) != FEPLB_OK) return 0;
+  return (size_t)c->T * c->K + (size_t)c->E * (c->row_align - 1);
+}
+
+extern "C" int feplb_select_dynamic(const int64_t* score, int32_t E, int32_t R, int32_t dyn, uint8_t* mask_out) {
+  if (!score || !mask_out || E < 1 || R < 1 || E % R || dyn < 0) return FEPLB_E_INVALID;
+  const int L = E / R;
+  // An expert is dynamic iff fewer than `dyn` experts of its block beat it
+  // (higher score, or equal score and lower id).
+  for (int e = 0; e < E; ++e) {
+    const int b0 = e / L * L;
+    int better = 0;
+    for (int o = b0; o < b0 + L; ++o)
+      better += (score[o] > score[e]) || (score[o] == score[e] && o < e);
+    mask_out[e] = better < dyn ? 1 : 0;
+  }
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_plan(const feplb_config* cfg, const int32_t* counts, const uint8_t* dyn_mask, feplb_plan_out* out) {
+  int rc = feplb_validate_config(cfg);
+  if (rc != FEPLB_OK) return rc;
+  if (!counts || !dyn_mask || !out || !out->load_before || !out->load_after) return FEPLB_E_INVALID;
+  if ((out->cap_moves > 0 && !out->moves) || (out->cap_groups > 0 && !out->groups)) return FEPLB_E_INVALID;
+  const int E = cfg->E, R = cfg->R, L = E / R;
+  const int D = cfg->ranks_per_domain > 0 ? cfg->ranks_per_domain : R;
+  const int64_t thr = std::max<int64_t>(cfg->tau, 1);
+  const int64_t g = cfg->split_granule;
+  const bool split = cfg->split != 0;
+  for (int e = 0; e < E; ++e)
+    if (counts[e] < 0) return FEPLB_E_INVALID;
+
+  std::vector<int64_t> load(R, 0), rem(E);
+  std::vector<int> used(R, 0);
+  std::vector<uint8_t> moved(E, 0);
+  std::vector<uint8_t> pair_used((size_t)E * R, 0);   // (expert, dst) already served
+  for (int e = 0; e < E; ++e) { rem[e] = counts[e]; load[e / L] += counts[e]; }
+  for (int r = 0; r < R; ++r) out->load_before[r] = load[r];
+
+  int n_moves = 0;
+  std::vector<int> cand;
+  cand.reserve(L);
+  for (int base = 0; base < R; base += D) {
+    int64_t total = 0;
+    for (int r = base; r < base + D; ++r) total += load[r];
+    const int64_t mean_up = (total + D - 1) / D;       // ceil of the domain's mean load
+    for (;;) {
+      // most loaded rank of the domain (lowest id on ties)
+      int src = base;
+      for (int r = base + 1; r < base + D; ++r)
+        if (load[r] > load[src]) src = r;
+      if (split && load[src] <= mean_up) break;
+      // least loaded rank that can still receive (lowest id on ties)
+      int dst = -1;
+      for (int r = base; r < base + D; ++r) {
+        if (r == src || used[r] >= cfg->max_num_dyn) continue;
+        if (split && load[r] >= mean_up) continue;
+        if (dst < 0 || load[r] < load[dst]) dst = r;
+      }
+      if (dst < 0) break;
+      const int64_t gap = load[src] - load[dst];
+      if (gap <= 0) break;
+      // eligible dynamic experts of the source, busiest first (lower id on ties)
+      cand.clear();
+      for (int e = src * L; e < (src + 1) * L; ++e)
+        if (dyn_mask[e] && !moved[e] && rem[e] >= thr && !pair_used[(size_t)e * R + dst]) cand.push_back(e);
+      std::stable_sort(cand.begin(), cand.end(), [&](int a, int b) { return rem[a] > rem[b]; });
+      int pick = -1;
+      int64_t rows = 0;
+      for (int e : cand) {
+        if (!split) {
+          if (rem[e] < gap) { pick = e; rows = rem[e]; break; }
+        } else {
+          int64_t m = std::min(rem[e], std::min(load[src] - mean_up, mean_up - load[dst]));
+          if (m < rem[e]) m = m / g * g;
+          if (m >= thr) { pick = e; rows = m; break; }
+        }
+        if (cfg->policy == FEPLB_POLICY_LITERAL) break;
+      }
+      if (pick < 0) break;
+      if (n_moves >= out->cap_moves) return FEPLB_E_NOMEM;
+      if (!split) moved[pick] = 1;
+      rem[pick] -= rows;
+      load[src] -= rows;
+      load[dst] += rows;
+      used[dst] += 1;
+      pair_used[(size_t)pick * R + dst] = 1;
+      out->moves[n_moves++] = feplb_move{pick, src, dst, (int32_t)rows};
+    }
+  }
+  out->n_moves = n_moves;
+  for (int r = 0; r < R; ++r) out->load_after[r] = load[r];
+
+  // Group table in expert order: moved pieces from the front of the segment, then the remainder.
+  const int A = cfg->row_align;
+  int n_groups = 0;
+  int64_t off = 0;
+  for (int e = 0; e < E; ++e) {
+    int64_t p = off;
+    for (int i = 0; i < n_moves; ++i) {
+      if (out->moves[i].expert != e) continue;
+      if (n_groups >= out->cap_groups) return FEPLB_E_NOMEM;
+      out->groups[n_groups++] = feplb_group{e, (int32_t)p, out->moves[i].rows, out->moves[i].dst, dyn_mask[e] ? 1 : 0};
+      p += out->moves[i].rows;
+    }
+    if (rem[e] > 0) {
+      if (n_groups >= out->cap_groups) return FEPLB_E_NOMEM;
+      out->groups[n_groups++] = feplb_group{e, (int32_t)p, (int32_t)rem[e], e / L, dyn_mask[e] ? 1 : 0};
+    }
+    off += ((int64_t)counts[e] + A - 1) / A * A;
+  }
+  out->n_groups = n_groups;
+  return FEPLB_OK;
+}

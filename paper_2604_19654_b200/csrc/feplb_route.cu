@@ -1,0 +1,302 @@
+// Integer side of the FEPLB hot path on sm_100a: routing histogram (paper Section 2.2: per-expert
+// token counts known after Phase 1), the stable counting-sort permutation of (token, k) slots
+// into expert-contiguous rows (Section 2.2: tokens "permuted" for the grouped GEMM), the row
+// gather, and the home (pre-plan) group table the static-expert GEMM runs on (Section 2.3).
+//
+// Ranks inside an expert's segment must not depend on the order in which atomics land, so
+// ranking is done in three deterministic levels: a warp ranks its 32 slots with match_any and
+// a lane mask, warps of a CTA are chained through per-warp histograms in shared memory, CTAs
+// are chained through an exclusive scan of per-CTA histograms.  Atomics are used only for the
+// per-expert totals (integer adds commute).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "feplb_internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunks = FEPLB_SLOTS_PER_BLOCK / kThreads;   // 32-slot chunks per warp (4)
+static_assert(FEPLB_SLOTS_PER_BLOCK == kWarps * kChunks * 32, "slot tiling");
+
+// Warp w of CTA b owns slots [b*1024 + w*128, +128) as kChunks chunks of 32 consecutive slots.
+// Fills the per-warp histograms wh[kWarps][E] and returns each lane's ids and match masks.
+__device__ __forceinline__ bool warp_histograms(const int32_t* __restrict__ ids, int64_t S, int E, int* wh,
+                                                int (&id)[kChunks], unsigned (&mk)[kChunks]) {
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < kWarps * E; i += kThreads) wh[i] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * FEPLB_SLOTS_PER_BLOCK + w * (kChunks * 32);
+  bool bad = false;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    const int64_t s = base + c * 32 + lane;
+    int v = -1;
+    if (s < S) {
+      v = ids[s];
+      if ((unsigned)v >= (unsigned)E) { bad = true; v = -1; }
+    }
+    id[c] = v;
+    mk[c] = __match_any_sync(0xffffffffu, v);
+    if (v >= 0 && lane == __ffs(mk[c]) - 1) wh[w * E + v] += __popc(mk[c]);
+    __syncwarp();
+  }
+  return bad;
+}
+
+// Step 1: per-CTA histograms; with counts != nullptr also the totals (one atomic per CTA and expert).
+__global__ void __launch_bounds__(kThreads)
+k_block_hist(const int32_t* __restrict__ ids, int64_t S, int E, int L, int32_t* __restrict__ block_hist,
+             int32_t* __restrict__ counts, int32_t* __restrict__ rank_load, uint32_t* status) {
+  extern __shared__ int wh[];
+  int id[kChunks];
+  unsigned mk[kChunks];
+  if (warp_histograms(ids, S, E, wh, id, mk)) atomicOr(status, FEPLB_ST_RANGE);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += kThreads) {
+    int sum = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) sum += wh[w * E + e];
+    if (block_hist) block_hist[(int64_t)blockIdx.x * E + e] = sum;
+    if (counts && sum) {
+      atomicAdd(&counts[e], sum);
+      atomicAdd(&rank_load[e / L], sum);
+    }
+  }
+}
+
+// Block-wide exclusive scan of v over threads 0..n-1 (n <= 1024 = blockDim.x); tmp holds 1024+32 ints.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* tmp, int* total) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) tmp[w] = x;
+  __syncthreads();
+  if (w == 0) {
+    int s = tmp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, s, o);
+      if (lane >= o) s += y;
+    }
+    tmp[32 + lane] = s;   // inclusive scan of the warp sums
+  }
+  __syncthreads();
+  const int warp_off = w ? tmp[32 + w - 1] : 0;
+  if (total) *total = tmp[32 + 31];
+  return warp_off + x - v;
+}
+
+// Exclusive scan of the per-CTA histograms over CTAs (in place), check against counts, and
+// pad_off[e] = sum_{e'<e} round_up(counts[e'], A); pad_off[E] = padded total.
+__global__ void __launch_bounds__(1024)
+k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __restrict__ counts,
+       int32_t* __restrict__ pad_off, uint32_t* status) {
+  __shared__ int tmp[64];
+  const int e = threadIdx.x;
+  int c = 0;
+  if (e < E) {
+    int run = 0;
+    for (int b = 0; b < nb; ++b) {
+      const int v = block_hist[(int64_t)b * E + e];
+      block_hist[(int64_t)b * E + e] = run;
+      run += v;
+    }
+    c = counts[e];
+    if (run != c) atomicOr(status, FEPLB_ST_COUNTS);
+  }
+  const int padded = (c + A - 1) / A * A;
+  int total;
+  const int off = block_exclusive_scan(padded, tmp, &total);
+  if (e < E) pad_off[e] = off;
+  if (e == 0) pad_off[E] = total;
+}
+
+// Stable rank of every slot: slot_to_row[s] and row_to_token[row].
+__global__ void __launch_bounds__(kThreads)
+k_rank(const int32_t* __restrict__ ids, int64_t S, int K, int E, const int32_t* __restrict__ block_base,
+       const int32_t* __restrict__ pad_off, int32_t* __restrict__ slot_to_row,
+       int32_t* __restrict__ row_to_token, int64_t s_cap) {
+  extern __shared__ int wh[];
+  int id[kChunks];
+  unsigned mk[kChunks];
+  warp_histograms(ids, S, E, wh, id, mk);
+  __syncthreads();
+  // chain the warps: wh[w][e] becomes the first row of warp w's slots of expert e
+  for (int e = threadIdx.x; e < E; e += kThreads) {
+    int run = pad_off[e] + block_base[(int64_t)blockIdx.x * E + e];
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const int t = wh[w * E + e];
+      wh[w * E + e] = run;
+      run += t;
+    }
+  }
+  __syncthreads();
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned lt = (1u << lane) - 1u;
+  const int64_t base = (int64_t)blockIdx.x * FEPLB_SLOTS_PER_BLOCK + w * (kChunks * 32);
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    const int64_t s = base + c * 32 + lane;
+    const int v = id[c];
+    int row = -1;
+    if (v >= 0) row = wh[w * E + v] + __popc(mk[c] & lt);
+    __syncwarp();
+    if (v >= 0 && lane == __ffs(mk[c]) - 1) wh[w * E + v] += __popc(mk[c]);
+    __syncwarp();
+    if (s < S) {
+      slot_to_row[s] = row;
+      if (row >= 0 && row < s_cap) row_to_token[row] = (int32_t)(s / K);
+    }
+  }
+}
+
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// Row gather, token-major: one warp reads a token's row once (16-byte vectors, coalesced) and
+// writes it to the K rows its slots were ranked to.
+constexpr int kGatherUnroll = 4;
+__global__ void __launch_bounds__(kThreads)
+k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, uint4* __restrict__ x_perm,
+         int T, int K, int chunks) {
+  const int lane = threadIdx.x & 31;
+  const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int nwarps = (gridDim.x * kThreads) >> 5;
+  for (int t = warp; t < T; t += nwarps) {
+    const int myrow = lane < K ? slot_to_row[(int64_t)t * K + lane] : -1;
+    const uint4* src = x + (int64_t)t * chunks;
+    for (int c0 = 0; c0 < chunks; c0 += 32 * kGatherUnroll) {
+      uint4 v[kGatherUnroll];
+#pragma unroll
+      for (int u = 0; u < kGatherUnroll; ++u) {
+        const int c = c0 + u * 32 + lane;
+        if (c < chunks) v[u] = ld_nc_v4(src + c);
+      }
+      for (int k = 0; k < K; ++k) {
+        const int row = __shfl_sync(0xffffffffu, myrow, k);
+        if (row < 0) continue;
+        uint4* dst = x_perm + (int64_t)row * chunks;
+#pragma unroll
+        for (int u = 0; u < kGatherUnroll; ++u) {
+          const int c = c0 + u * 32 + lane;
+          if (c < chunks) dst[c] = v[u];
+        }
+      }
+    }
+  }
+}
+
+// Zero the padding rows at the end of every expert's segment (row_align > 1 only).
+__global__ void __launch_bounds__(kThreads)
+k_zero_pad(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_off, uint4* __restrict__ x_perm,
+           int chunks) {
+  const int e = blockIdx.x;
+  const int64_t r0 = (int64_t)pad_off[e] + counts[e], r1 = pad_off[e + 1];
+  const int64_t n = (r1 - r0) * chunks;
+  uint4* p = x_perm + r0 * chunks;
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  for (int64_t i = threadIdx.x; i < n; i += kThreads) p[i] = z;
+}
+
+// Home group table {e, pad_off[e], counts[e], home(e), dynamic?} for all E experts.
+__global__ void __launch_bounds__(1024)
+k_home_groups(const int32_t* __restrict__ counts, const uint8_t* __restrict__ mask_in, int E, int L, int A, int dyn,
+              feplb_group* __restrict__ groups, uint8_t* __restrict__ mask_out) {
+  __shared__ int tmp[64];
+  __shared__ int sc[FEPLB_MAX_EXPERTS];
+  const int e = threadIdx.x;
+  const int c = e < E ? counts[e] : 0;
+  if (e < E) sc[e] = c;
+  const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, nullptr);
+  if (e >= E) return;
+  int is_dyn;
+  if (mask_in) {
+    is_dyn = mask_in[e] != 0;
+  } else {
+    // dynamic iff fewer than `dyn` experts of the block are busier (ties: lower id is busier)
+    const int b0 = e / L * L;
+    int better = 0;
+    for (int o = b0; o < b0 + L; ++o) better += (sc[o] > c) || (sc[o] == c && o < e);
+    is_dyn = better < dyn;
+  }
+  groups[e] = feplb_group{e, off, c, e / L, is_dyn};
+  if (mask_out) mask_out[e] = (uint8_t)is_dyn;
+}
+
+}  // namespace
+
+cudaError_t feplb_launch_block_hist(const int32_t* ids, int64_t S, int E, int R, int32_t* block_hist,
+                                    int32_t* counts, int32_t* rank_load, uint32_t* status,
+                                    cudaStream_t st, int64_t* n_launch) {
+  cudaError_t err;
+  if (counts) {
+    if ((err = cudaMemsetAsync(counts, 0, sizeof(int32_t) * E, st)) != cudaSuccess) return err;
+    if ((err = cudaMemsetAsync(rank_load, 0, sizeof(int32_t) * R, st)) != cudaSuccess) return err;
+  }
+  const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
+  if (nb == 0) return cudaSuccess;
+  k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E / R, block_hist, counts, rank_load, status);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, int A, const int32_t* counts,
+                                 int32_t* block_hist, int32_t* pad_off, int32_t* slot_to_row,
+                                 int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                 cudaStream_t st, int64_t* n_launch) {
+  cudaError_t err;
+  const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
+  if (s_cap > 0 && (err = cudaMemsetAsync(row_to_token, 0xFF, sizeof(int32_t) * s_cap, st)) != cudaSuccess) return err;
+  if (nb) {
+    k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E, block_hist, nullptr, nullptr, status);
+    ++*n_launch;
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  k_scan<<<1, 1024, 0, st>>>(block_hist, nb, E, A, counts, pad_off, status);
+  ++*n_launch;
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if (nb) {
+    k_rank<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, K, E, block_hist, pad_off, slot_to_row, row_to_token, s_cap);
+    ++*n_launch;
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
+                                const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
+                                cudaStream_t st, int64_t* n_launch) {
+  cudaError_t err;
+  const int chunks = d / 8;
+  if (A > 1) {
+    k_zero_pad<<<E, kThreads, 0, st>>>(counts, pad_off, (uint4*)x_perm, chunks);
+    ++*n_launch;
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  if (T == 0) return cudaSuccess;
+  const int warps_per_block = kThreads / 32;
+  int blocks = (T + warps_per_block - 1) / warps_per_block;
+  const int max_blocks = 148 * 8;
+  if (blocks > max_blocks) blocks = max_blocks;
+  k_gather<<<blocks, kThreads, 0, st>>>((const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
+                                     feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch) {
+  k_home_groups<<<1, 1024, 0, st>>>(counts, mask_in, E, E / R, A, dyn, groups, mask_out);
+  ++*n_launch;
+  return cudaGetLastError();
+}

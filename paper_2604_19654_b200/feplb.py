@@ -1,0 +1,322 @@
+"""Thin ctypes binding over the C ABI of ``libfeplb.so`` (see ``include/feplb.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels (or, for
+the plan, in its C++ host code).  PyTorch supplies device memory and streams.  If the library is
+missing the import of a symbol fails loudly -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfeplb.so")
+
+OK, E_INVALID, E_RANGE, E_CUDA, E_NOMEM, E_TIMEOUT, E_STATE, E_DEVICE = 0, -1, -2, -3, -4, -5, -6, -7
+POLICY_LITERAL, POLICY_FIRST_FIT = 0, 1
+MASK_GIVEN, MASK_REACTIVE = 0, 1
+FFN_ALL, FFN_STATIC, FFN_DYNAMIC = 0, 1, 2
+
+
+class Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "T", "K", "E", "R", "d", "f", "dyn", "max_num_dyn", "tau", "ranks_per_domain", "policy",
+        "split", "split_granule", "row_align", "mask_policy")]
+
+
+class Move(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("expert", "src", "dst", "rows")]
+
+
+class Group(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("expert", "row_start", "rows", "exec_rank", "is_dynamic")]
+
+
+class PlanOut(C.Structure):
+    _fields_ = [("n_moves", C.c_int32), ("n_groups", C.c_int32), ("cap_moves", C.c_int32),
+                ("cap_groups", C.c_int32), ("moves", C.POINTER(Move)), ("groups", C.POINTER(Group)),
+                ("load_before", C.POINTER(C.c_int64)), ("load_after", C.POINTER(C.c_int64))]
+
+
+class Timeline(C.Structure):
+    _fields_ = [(n, C.c_double) for n in (
+        "host_enqueue_static_done_us", "host_counts_ready_us", "host_plan_done_us",
+        "host_upload_enqueued_us", "host_join_us", "host_return_us", "plan_us",
+        "dev_hist_us", "dev_dispatch_us", "dev_static_ffn_us", "dev_dynamic_ffn_us", "dev_combine_us",
+        "dev_counts_to_static_start_us", "dev_counts_to_static_end_us", "dev_total_us")]
+
+
+class FeplbError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {lib().feplb_strerror(code).decode()} ({code})" + (f": {detail}" if detail else ""))
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Opens libfeplb.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2604_19654_b200.build` "
+                "(the CUDA library is the only implementation; there is no fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        sig = {
+            "feplb_version": (C.c_int, []),
+            "feplb_strerror": (C.c_char_p, [C.c_int]),
+            "feplb_create": (C.c_int, [C.POINTER(Config), C.POINTER(vp)]),
+            "feplb_destroy": (C.c_int, [vp]),
+            "feplb_last_error": (C.c_char_p, [vp]),
+            "feplb_check_status": (C.c_int, [vp, vp]),
+            "feplb_s_pad": (C.c_size_t, [C.POINTER(Config)]),
+            "feplb_select_dynamic": (C.c_int, [C.POINTER(i64), i32, i32, i32, C.POINTER(C.c_uint8)]),
+            "feplb_plan": (C.c_int, [C.POINTER(Config), C.POINTER(i32), C.POINTER(C.c_uint8), C.POINTER(PlanOut)]),
+            "feplb_route_hist": (C.c_int, [vp, vp, vp, vp, vp]),
+            "feplb_dispatch": (C.c_int, [vp] * 8),
+            "feplb_home_groups": (C.c_int, [vp] * 6),
+            "feplb_expert_ffn": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
+            "feplb_combine": (C.c_int, [vp] * 6),
+            "feplb_plan_async": (C.c_int, [vp, vp, vp, vp]),
+            "feplb_plan_wait": (C.c_int, [vp, i32, C.POINTER(PlanOut), C.POINTER(vp), C.POINTER(i32), vp]),
+            "feplb_moe_forward": (C.c_int, [vp] * 16 + [C.POINTER(PlanOut), vp]),
+            "feplb_moe_forward_host": (C.c_int, [vp] * 20 + [C.POINTER(PlanOut), vp]),
+            "feplb_set_timeline": (C.c_int, [vp, i32]),
+            "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
+            "feplb_launch_count": (i64, [vp]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def make_config(T, K, E, R, d, f, dyn=4, max_num_dyn=8, tau=0, ranks_per_domain=0,
+                policy=POLICY_FIRST_FIT, split=0, split_granule=128, row_align=1,
+                mask_policy=MASK_REACTIVE) -> Config:
+    return Config(T, K, E, R, d, f, dyn, max_num_dyn, tau, ranks_per_domain, policy, split,
+                  split_granule, row_align, mask_policy)
+
+
+def config_from_workload(w, **kw) -> Config:
+    base = dict(T=w.T, K=w.K, E=w.E, R=w.R, d=w.d, f=w.f, dyn=w.dyn, max_num_dyn=w.max_num_dyn, tau=w.tau)
+    base.update(kw)
+    return make_config(**base)
+
+
+def s_pad(cfg: Config) -> int:
+    return int(lib().feplb_s_pad(C.byref(cfg)))
+
+
+class Plan:
+    """Host copy of a plan: moves, groups, per-rank loads (numpy)."""
+
+    def __init__(self, cfg: Config):
+        self.cap_moves = max(1, cfg.R * cfg.max_num_dyn)
+        self.cap_groups = cfg.E + cfg.R * cfg.max_num_dyn
+        self._moves = (Move * self.cap_moves)()
+        self._groups = (Group * self.cap_groups)()
+        self._lb = (C.c_int64 * cfg.R)()
+        self._la = (C.c_int64 * cfg.R)()
+        self.c = PlanOut(0, 0, self.cap_moves, self.cap_groups, self._moves, self._groups, self._lb, self._la)
+
+    @property
+    def moves(self):
+        return [(m.expert, m.src, m.dst, m.rows) for m in self._moves[: self.c.n_moves]]
+
+    @property
+    def groups(self):
+        return [(g.expert, g.row_start, g.rows, g.exec_rank, g.is_dynamic) for g in self._groups[: self.c.n_groups]]
+
+    @property
+    def load_before(self):
+        return np.array(self._lb[:], np.int64)
+
+    @property
+    def load_after(self):
+        return np.array(self._la[:], np.int64)
+
+
+def select_dynamic(score: Sequence[int], E: int, R: int, dyn: int) -> np.ndarray:
+    sc = np.ascontiguousarray(score, np.int64)
+    out = np.zeros(E, np.uint8)
+    rc = lib().feplb_select_dynamic(sc.ctypes.data_as(C.POINTER(C.c_int64)), E, R, dyn,
+                                    out.ctypes.data_as(C.POINTER(C.c_uint8)))
+    if rc:
+        raise FeplbError(rc, "feplb_select_dynamic")
+    return out
+
+
+def plan(cfg: Config, counts, dyn_mask) -> Plan:
+    """Host-only greedy plan (no GPU needed)."""
+    cnt = np.ascontiguousarray(counts, np.int32)
+    msk = np.ascontiguousarray(dyn_mask, np.uint8)
+    if cnt.shape != (cfg.E,) or msk.shape != (cfg.E,):
+        raise ValueError("counts and dyn_mask must have E entries")
+    p = Plan(cfg)
+    rc = lib().feplb_plan(C.byref(cfg), cnt.ctypes.data_as(C.POINTER(C.c_int32)),
+                          msk.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(p.c))
+    if rc:
+        raise FeplbError(rc, "feplb_plan")
+    return p
+
+
+def _ptr(t) -> Optional[int]:
+    """Device/host address of a torch tensor or numpy array (None passes NULL)."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def groups_to_numpy(groups) -> np.ndarray:
+    """[(expert, row_start, rows, exec_rank, is_dynamic)] -> int32 [n, 5] in the ABI's struct layout."""
+    a = np.asarray(groups, np.int32).reshape(-1, 5)
+    return np.ascontiguousarray(a)
+
+
+class Context:
+    """One layer geometry on the current CUDA device.  Calls on one context must not overlap."""
+
+    def __init__(self, cfg: Config):
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        rc = lib().feplb_create(C.byref(cfg), C.byref(self._h))
+        if rc:
+            raise FeplbError(rc, "feplb_create")
+        self.s_cap = s_pad(cfg)
+
+    def close(self):
+        if self._h:
+            lib().feplb_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _chk(self, rc, where):
+        if rc:
+            raise FeplbError(rc, where, lib().feplb_last_error(self._h).decode())
+
+    @staticmethod
+    def _stream(stream) -> Optional[int]:
+        if stream is None:
+            import torch
+            return torch.cuda.current_stream().cuda_stream or None
+        return getattr(stream, "cuda_stream", stream) or None
+
+    def check_status(self, stream=None):
+        self._chk(lib().feplb_check_status(self._h, self._stream(stream)), "feplb_check_status")
+
+    def route_hist(self, topk_ids, counts, rank_load, stream=None):
+        self._chk(lib().feplb_route_hist(self._h, _ptr(topk_ids), _ptr(counts), _ptr(rank_load),
+                                         self._stream(stream)), "feplb_route_hist")
+
+    def dispatch(self, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, stream=None):
+        self._chk(lib().feplb_dispatch(self._h, _ptr(x), _ptr(topk_ids), _ptr(counts), _ptr(x_perm),
+                                       _ptr(slot_to_row), _ptr(row_to_token), self._stream(stream)), "feplb_dispatch")
+
+    def home_groups(self, counts, dyn_mask, groups_out, dyn_mask_out=None, stream=None):
+        self._chk(lib().feplb_home_groups(self._h, _ptr(counts), _ptr(dyn_mask), _ptr(groups_out),
+                                          _ptr(dyn_mask_out), self._stream(stream)), "feplb_home_groups")
+
+    def expert_ffn(self, x_perm, w1, w3, w2, groups, n_groups, h_scratch, y_perm, which=FFN_ALL, stream=None):
+        self._chk(lib().feplb_expert_ffn(self._h, _ptr(x_perm), _ptr(w1), _ptr(w3), _ptr(w2), _ptr(groups),
+                                         int(n_groups), int(which), _ptr(h_scratch), _ptr(y_perm),
+                                         self._stream(stream)), "feplb_expert_ffn")
+
+    def combine(self, y_perm, slot_to_row, gates, out, stream=None):
+        self._chk(lib().feplb_combine(self._h, _ptr(y_perm), _ptr(slot_to_row), _ptr(gates), _ptr(out),
+                                      self._stream(stream)), "feplb_combine")
+
+    def plan_async(self, counts, dyn_mask_host=None, stream=None):
+        self._mask_keepalive = None if dyn_mask_host is None else np.ascontiguousarray(dyn_mask_host, np.uint8)
+        self._chk(lib().feplb_plan_async(self._h, _ptr(counts), _ptr(self._mask_keepalive), self._stream(stream)),
+                  "feplb_plan_async")
+
+    def plan_wait(self, timeout_ms=2000, stream=None):
+        """Returns (Plan, device address of the dynamic group table, number of dynamic groups)."""
+        p = Plan(self.cfg)
+        dev = C.c_void_p()
+        n = C.c_int32()
+        self._chk(lib().feplb_plan_wait(self._h, int(timeout_ms), C.byref(p.c), C.byref(dev), C.byref(n),
+                                        self._stream(stream)), "feplb_plan_wait")
+        return p, dev.value, n.value
+
+    def moe_forward(self, x, topk_ids, gates, w1, w3, w2, buf, dyn_mask_host=None, want_plan=True, stream=None):
+        """``buf``: object with counts, rank_load, x_perm, h_scratch, y_perm, slot_to_row, row_to_token, out."""
+        p = Plan(self.cfg) if want_plan else None
+        mask = None if dyn_mask_host is None else np.ascontiguousarray(dyn_mask_host, np.uint8)
+        self._chk(lib().feplb_moe_forward(
+            self._h, _ptr(x), _ptr(topk_ids), _ptr(gates), _ptr(w1), _ptr(w3), _ptr(w2), _ptr(mask),
+            _ptr(buf.counts), _ptr(buf.rank_load), _ptr(buf.x_perm), _ptr(buf.h_scratch), _ptr(buf.y_perm),
+            _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(buf.out),
+            C.byref(p.c) if p is not None else None, self._stream(stream)), "feplb_moe_forward")
+        return p
+
+    def moe_forward_host(self, x_host, ids_host, gates_host, x_dev, ids_dev, gates_dev, w1, w3, w2, buf, out_host,
+                         dyn_mask_host=None, want_plan=False, stream=None):
+        p = Plan(self.cfg) if want_plan else None
+        mask = None if dyn_mask_host is None else np.ascontiguousarray(dyn_mask_host, np.uint8)
+        self._chk(lib().feplb_moe_forward_host(
+            self._h, _ptr(x_host), _ptr(ids_host), _ptr(gates_host), _ptr(x_dev), _ptr(ids_dev), _ptr(gates_dev),
+            _ptr(w1), _ptr(w3), _ptr(w2), _ptr(mask),
+            _ptr(buf.counts), _ptr(buf.rank_load), _ptr(buf.x_perm), _ptr(buf.h_scratch), _ptr(buf.y_perm),
+            _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(buf.out), _ptr(out_host),
+            C.byref(p.c) if p is not None else None, self._stream(stream)), "feplb_moe_forward_host")
+        return p
+
+    def set_timeline(self, on: bool):
+        self._chk(lib().feplb_set_timeline(self._h, int(bool(on))), "feplb_set_timeline")
+
+    def get_timeline(self) -> dict:
+        t = Timeline()
+        self._chk(lib().feplb_get_timeline(self._h, C.byref(t)), "feplb_get_timeline")
+        return {n: getattr(t, n) for n, _ in Timeline._fields_}
+
+    def launch_count(self) -> int:
+        return int(lib().feplb_launch_count(self._h))
+
+
+class Buffers:
+    """Caller-owned device outputs and scratch of one layer geometry (torch tensors on ``device``)."""
+
+    def __init__(self, cfg: Config, device="cuda"):
+        import torch
+        cap = s_pad(cfg)
+        i32, bf = torch.int32, torch.bfloat16
+        self.counts = torch.zeros(cfg.E, dtype=i32, device=device)
+        self.rank_load = torch.zeros(cfg.R, dtype=i32, device=device)
+        self.x_perm = torch.empty(max(cap, 1), cfg.d, dtype=bf, device=device)
+        self.h_scratch = torch.empty(max(cap, 1), cfg.f, dtype=bf, device=device)
+        self.y_perm = torch.empty(max(cap, 1), cfg.d, dtype=bf, device=device)
+        self.slot_to_row = torch.empty(max(cfg.T, 1), cfg.K, dtype=i32, device=device)
+        self.row_to_token = torch.empty(max(cap, 1), dtype=i32, device=device)
+        self.out = torch.empty(max(cfg.T, 1), cfg.d, dtype=bf, device=device)
+
+
+def bf16_tensor(bits: np.ndarray, device="cuda"):
+    """numpy uint16 bf16 bit patterns -> torch.bfloat16 tensor on ``device`` (bit copy)."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    return t.to(device)
+
+
+def bf16_bits(t) -> np.ndarray:
+    """torch.bfloat16 tensor -> numpy uint16 bit patterns (bit copy)."""
+    import torch
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)

@@ -1,0 +1,126 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, and
+its host-only steps (plan, dynamic-expert selection, sizing, argument checks) agree bit-exactly
+with the oracle.  No compute call touches a GPU here."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+from oracle import feplb_oracle as O
+from paper_2604_19654_b200 import build as B
+from paper_2604_19654_b200 import feplb as F
+from paper_2604_19654_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    B.build()
+
+
+def _declared_symbols():
+    names = []
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names += re.findall(r"\b(feplb_[a-z0-9_]+)\s*\(", src)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_symbols()
+    assert len(names) >= 20 and "feplb_expert_ffn" in names
+    L = C.CDLL(F.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+    assert F.lib().feplb_version() >= 100
+    assert F.lib().feplb_strerror(F.E_TIMEOUT) == b"timed out"
+
+
+def test_config_validation_and_s_pad():
+    cfg = F.make_config(T=256, K=2, E=8, R=2, d=128, f=64)
+    assert F.s_pad(cfg) == 512
+    cfg128 = F.make_config(T=256, K=2, E=8, R=2, d=128, f=64, row_align=128)
+    assert F.s_pad(cfg128) == 512 + 8 * 127
+    for bad in (dict(E=7), dict(d=100), dict(f=32), dict(K=0), dict(K=33), dict(row_align=64), dict(R=3),
+                dict(ranks_per_domain=3), dict(policy=7), dict(split_granule=0)):
+        kw = dict(T=256, K=2, E=8, R=2, d=128, f=64)
+        kw.update(bad)
+        c = F.make_config(**kw)
+        assert F.s_pad(c) == 0
+        with pytest.raises(F.FeplbError):
+            F.plan(c, np.zeros(c.E, np.int32), np.zeros(c.E, np.uint8))
+
+
+def test_create_without_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(F.FeplbError):
+        F.Context(F.make_config(T=256, K=2, E=8, R=2, d=128, f=64))
+
+
+def _same_plan(cfg, counts, mask, A=1):
+    p = F.plan(cfg, counts, mask)
+    o = O.plan(counts, mask, cfg.R, tau=cfg.tau, max_num_dyn=cfg.max_num_dyn,
+               ranks_per_domain=cfg.ranks_per_domain, policy=cfg.policy, split=cfg.split,
+               split_granule=cfg.split_granule, row_align=A)
+    assert p.moves == [tuple(int(v) for v in m) for m in o["moves"]]
+    assert p.groups == [tuple(int(v) for v in g) for g in o["groups"]]
+    assert np.array_equal(p.load_before, o["load_before"])
+    assert np.array_equal(p.load_after, o["load_after"])
+    return p
+
+
+@settings(max_examples=400, deadline=None)
+@given(st.sampled_from([1, 2, 3, 4, 8, 16]), st.integers(1, 8), st.integers(0, 2 ** 31),
+       st.sampled_from([0, 1, 5, 64]), st.integers(0, 8), st.sampled_from([0, 1]), st.sampled_from([0, 1]),
+       st.sampled_from([1, 16, 128]), st.booleans(), st.sampled_from([1, 128]))
+def test_plan_matches_oracle_bit_exact(R, L, seed, tau, mnd, policy, split, g, dom, A):
+    rng = np.random.default_rng(seed)
+    E = R * L
+    scale = int(rng.choice([3, 50, 1500]))
+    counts = (rng.dirichlet(np.full(E, 0.3)) * scale * E).astype(np.int32)
+    mask = (rng.random(E) < 0.6).astype(np.uint8)
+    D = 2 if (dom and R % 2 == 0) else 0
+    cfg = F.make_config(T=1, K=1, E=E, R=R, d=128, f=64, max_num_dyn=mnd, tau=tau, ranks_per_domain=D,
+                        policy=policy, split=split, split_granule=g, row_align=A)
+    _same_plan(cfg, counts, mask, A)
+
+
+def test_plan_matches_oracle_on_workloads():
+    for name in ("cfg1", "cfg2", "cfg3", "cfg3-smooth", "cfg4"):
+        w = W.get_workload(name)
+        for mb in range(min(3, w.n_microbatches)):
+            ids, _ = W.gen_routing(w, mb)
+            counts, _ = O.route_hist(ids, w.E, w.R)
+            mask = O.select_dynamic(counts, w.E, w.R, w.dyn)
+            assert np.array_equal(F.select_dynamic(counts, w.E, w.R, w.dyn), mask)
+            for split in (0, 1):
+                for policy in (0, 1):
+                    cfg = F.config_from_workload(w, split=split, policy=policy)
+                    _same_plan(cfg, counts.astype(np.int32), mask)
+
+
+@settings(max_examples=100, deadline=None)
+@given(st.sampled_from([1, 2, 4]), st.integers(1, 9), st.integers(0, 10), st.integers(0, 2 ** 31))
+def test_select_dynamic_matches_oracle(R, L, dyn, seed):
+    rng = np.random.default_rng(seed)
+    score = rng.integers(0, 6, size=R * L)                     # many ties
+    assert np.array_equal(F.select_dynamic(score, R * L, R, dyn), O.select_dynamic(score, R * L, R, dyn))
+
+
+def test_plan_capacity_error():
+    cfg = F.make_config(T=1, K=1, E=4, R=2, d=128, f=64, max_num_dyn=2, tau=1)
+    p = F.Plan(cfg)
+    p.c.cap_groups = 1
+    cnt = np.array([50, 5, 1, 1], np.int32)
+    msk = np.ones(4, np.uint8)
+    rc = F.lib().feplb_plan(C.byref(cfg), cnt.ctypes.data_as(C.POINTER(C.c_int32)),
+                            msk.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(p.c))
+    assert rc == F.E_NOMEM
