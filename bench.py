@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the FEPLB MoE-layer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+A step is one pass of the whole path (route_hist -> plan || dispatch + static FFN -> dynamic FFN
+-> combine) over one seeded synthetic micro-batch.  Rank 0 prints ONE JSON line.  With N > 1
+(torchrun) every rank runs its own micro-batches, there is no data-path collective, and the value
+is all ranks' tokens over the slowest rank's device time (weak scaling).
+
+``--impl reference`` times the CPU oracle (oracle/), as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_19654_b200 import workloads as W  # noqa: E402
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+# DRAM bytes (read + write) of one k_grouped_gemm launch at the benchmarked workload, from the ncu
+# capture summarised under profiles/; None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm_gbs=j["hbm_gbs"], bf16_tflops=j["bf16_tflops"],
+                    bf16_tflops_sustained=j.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [s.strip() for s in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- oracle arm
+
+def _oracle_step(O, w, x, ids, gates, weights, tokens):
+    """The oracle's whole path on the micro-batch restricted to ``tokens``."""
+    sub_ids, sub_x, sub_g = ids[tokens], x[tokens], gates[tokens]
+    counts, load = O.route_hist(sub_ids, w.E, w.R)
+    mask = O.select_dynamic(counts, w.E, w.R, w.dyn)
+    plan = O.plan(counts, mask, w.R, tau=w.tau, max_num_dyn=w.max_num_dyn)
+    s2r, r2t, _, S_pad = O.permute(sub_ids, w.E, 1)
+    xp = O.gather_rows(sub_x, r2t)
+    y = O.expert_ffn(xp, O.row_experts(sub_ids, s2r, S_pad), *weights)
+    out = O.combine(y, s2r, sub_g)
+    return out, plan
+
+
+def _oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(w, steps, warmup, sample_tokens, weights=None):
+    from oracle import feplb_oracle as O
+    weights = weights if weights is not None else W.gen_weights(w)
+    times = []
+    for i in range(warmup + steps):
+        x, ids, gates = W.gen_microbatch(w, i % w.n_microbatches)
+        tokens = np.arange(min(sample_tokens, w.T))
+        t0 = time.perf_counter()
+        _oracle_step(O, w, x, ids, gates, weights, tokens)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    n_tok = min(sample_tokens, w.T)
+    return n_tok * len(times) / sum(times), 1e3 * sum(times) / len(times), n_tok
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = min(w.T, args.ref_sample_tokens)
+    val, ms, n_tok = time_oracle(w, args.steps, args.warmup, sample)
+    cores = _oracle_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": _config_dict(w, args, extra={"sample_tokens_per_step": n_tok}),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {n_tok} tokens of each micro-batch, whole path (numpy fp64 oracle)"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def _config_dict(w, args, extra=None):
+    c = {"workload": w.name, "T": w.T, "d": w.d, "f": w.f, "E": w.E, "top_k": w.K, "virtual_ranks": w.R,
+         "dyn": w.dyn, "max_num_dyn": w.max_num_dyn, "tau": w.tau, "micro_batches": w.n_microbatches,
+         "routing": f"{w.routing}(alpha={w.alpha})", "parallelism": f"dp{args.gpus} (independent micro-batches per rank)",
+         "cache": "inputs rotate over the micro-batches; weights (%.2f GiB) exceed the 126 MB L2"
+                  % (3 * w.E * w.d * w.f * 2 / 2 ** 30)}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# --------------------------------------------------------------------------------------------- CUDA arm
+
+def gemm_flops(w):
+    """Algorithmic flops of the expert FFN per micro-batch: three GEMMs, 2*d*f each, per slot."""
+    return 6.0 * w.d * w.f * w.S
+
+
+def run_cuda(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_19654_b200 import build as B
+    from paper_2604_19654_b200 import feplb as F
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.build()
+    cfg = F.config_from_workload(w)
+    ctx = F.Context(cfg)
+    buf = F.Buffers(cfg)
+
+    weights = W.gen_weights(w)
+    d_w1, d_w3, d_w2 = (F.bf16_tensor(a) for a in weights)
+    n_mb = w.n_microbatches
+    host = [W.gen_microbatch(w, rank * n_mb + i) for i in range(n_mb)]      # every rank its own micro-batches
+    dev = [(F.bf16_tensor(x), torch.from_numpy(i).cuda(), torch.from_numpy(g).cuda()) for x, i, g in host]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        x, ids, g = dev[i % n_mb]
+        ctx.moe_forward(x, ids, g, d_w1, d_w3, d_w2, buf, want_plan=False, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    ctx.check_status()
+    ctx.set_timeline(True)
+    ctx.timeline_totals(reset=True)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches0 = ctx.launch_count()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev0.elapsed_time(ev1)
+    totals, n_fw = ctx.timeline_totals(reset=True)
+    ctx.set_timeline(False)
+    ctx.check_status()
+    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    value = world * args.steps * w.T / (ms_total * 1e-3)
+
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    pinned = []
+    for x, i, g in host:
+        pinned.append((torch.from_numpy(x.view(np.int16)).pin_memory(), torch.from_numpy(i).pin_memory(),
+                       torch.from_numpy(g).pin_memory()))
+    out_host = torch.empty(w.T, w.d, dtype=torch.int16).pin_memory()
+    x_dev = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    i_dev = torch.empty(w.T, w.K, dtype=torch.int32, device="cuda")
+    g_dev = torch.empty(w.T, w.K, dtype=torch.float32, device="cuda")
+
+    def step_host(i):
+        xh, ih, gh = pinned[i % n_mb]
+        ctx.moe_forward_host(xh, ih, gh, x_dev, i_dev, g_dev, d_w1, d_w3, d_w2, buf, out_host, stream=stream)
+
+    for i in range(3):
+        step_host(i)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step_host(i)
+    e1.record(stream)
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), 0.0)
+    del t0
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * args.steps * w.T / (float(t.item()) * 1e-3)
+    h2d = w.T * w.d * 2 + 2 * w.T * w.K * 4
+    d2h = w.T * w.d * 2
+
+    # ---- stragglers: token loads from the plan; GEMM time of every virtual rank run alone ---------
+    strag = None
+    if rank == 0 and not args.no_straggler:
+        strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb)
+
+    if rank == 0:
+        peaks = _peaks()
+        ffn_us = totals["dev_static_ffn_us"] + totals["dev_dynamic_ffn_us"]
+        gemm_launches = 4 * n_fw
+        flops_launch = gemm_flops(w) / 4.0
+        achieved = (flops_launch / (ffn_us * 1e-6 / gemm_launches)) / 1e12 if ffn_us > 0 else None
+        # a kernel timed inside a long step: the sustained bf16 figure is the honest denominator
+        peak = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
+        io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
+        roof = {"bound": "tensor", "kernel": "k_grouped_gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak if achieved else None, "peak_source": peaks["source"] + " (sustained)",
+                "frac_of_burst": achieved / peaks["bf16_tflops"] if achieved else None,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                "launches_timed": gemm_launches, "avg_launch_us": ffn_us / gemm_launches if gemm_launches else None,
+                "dispatch_gbs": io_bytes / (totals["dev_dispatch_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_dispatch_us"] else None,
+                "combine_gbs": io_bytes / (totals["dev_combine_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_combine_us"] else None,
+                "hbm_peak_gbs": peaks["hbm_gbs"]}
+        stage_us = {k: (v / n_fw if n_fw else None) for k, v in totals.items()}
+        # CPU oracle on the host cores: a bounded sample of the same workload
+        cpu_val, cpu_ms, n_tok = time_oracle(w, 2, 1, min(w.T, 4096), weights)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": _config_dict(w, args),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
+            "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+                             "sample": f"first {n_tok} tokens of 2 micro-batches, whole path (numpy fp64 oracle)"},
+            "stage_us": stage_us, "straggler": strag,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb, reps=3):
+    """Token straggler from the plans and GEMM straggler from per-virtual-rank launches, before
+    (every group on its home rank) and after rebalancing, averaged over the micro-batches."""
+    import torch
+    tok_b, tok_a, gem_b, gem_a, gem_bm, gem_am = [], [], [], [], [], []
+    L = w.E // w.R
+    for i in range(min(n_mb, 4)):
+        x, ids, g = dev[i]
+        p = ctx.moe_forward(x, ids, g, d_w1, d_w3, d_w2, buf, want_plan=True, stream=stream)
+        torch.cuda.synchronize()
+        lb, la = p.load_before.astype(np.float64), p.load_after.astype(np.float64)
+        tok_b.append(lb.max() / lb.mean())
+        tok_a.append(la.max() / la.mean())
+        groups = p.groups
+        per_rank = {"before": [], "after": []}
+        for label, key in (("before", lambda gr: gr[0] // L), ("after", lambda gr: gr[3])):
+            for r in range(w.R):
+                sel = [gr for gr in groups if key(gr) == r]
+                if not sel:
+                    per_rank[label].append(0.0)
+                    continue
+                d_groups = torch.from_numpy(F.groups_to_numpy(sel)).cuda()
+                ts = []
+                for _ in range(reps):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    ctx.expert_ffn(buf.x_perm, d_w1, d_w3, d_w2, d_groups, len(sel), buf.h_scratch, buf.y_perm, stream=stream)
+                    e1.record(stream)
+                    torch.cuda.synchronize()
+                    ts.append(e0.elapsed_time(e1))
+                per_rank[label].append(float(np.median(ts)))
+        b, a = np.array(per_rank["before"]), np.array(per_rank["after"])
+        gem_b.append(b.max() / b.mean())
+        gem_a.append(a.max() / a.mean())
+        gem_bm.append(b.max() - b.mean())
+        gem_am.append(a.max() - a.mean())
+    return {"token_ratio_before": float(np.mean(tok_b)), "token_ratio_after": float(np.mean(tok_a)),
+            "gemm_ratio_before": float(np.mean(gem_b)), "gemm_ratio_after": float(np.mean(gem_a)),
+            "gemm_max_minus_mean_ms_before": float(np.mean(gem_bm)), "gemm_max_minus_mean_ms_after": float(np.mean(gem_am)),
+            "micro_batches": len(tok_b), "definition": "max over virtual ranks / mean; GEMM time = expert FFN of one rank's groups run alone"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--ref-sample-tokens", type=int, default=1024)
+    ap.add_argument("--no-straggler", action="store_true")
+    args = ap.parse_args()
+    w = W.get_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

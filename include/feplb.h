@@ -229,8 +229,13 @@ int feplb_moe_forward_host(feplb_ctx* ctx, const void* x_host, const int32_t* to
 
 /* Turns CUDA-event timing of the stages of feplb_moe_forward on (1) or off (0, default). */
 int feplb_set_timeline(feplb_ctx* ctx, int32_t enable);
-/* Synchronises the last forward's events and fills *out (device fields are 0 when disabled). */
+/* Waits for the last forward's stage events and fills *out (device fields are 0 when timing was
+ * off during that forward). */
 int feplb_get_timeline(feplb_ctx* ctx, feplb_timeline* out);
+/* Sums of every field over the forwards run with timing on since the last reset, and their
+ * number.  The stage events of up to 16 forwards stay outstanding, so timing does not make the
+ * host wait for the GPU between forwards; this call waits for the outstanding ones. */
+int feplb_timeline_totals(feplb_ctx* ctx, feplb_timeline* sum, int64_t* n_forwards, int32_t reset);
 /* Number of kernels this library has launched on `ctx` since creation. */
 int64_t feplb_launch_count(const feplb_ctx* ctx);
 

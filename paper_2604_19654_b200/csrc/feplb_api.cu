@@ -22,7 +22,8 @@ inline double us_since(clk::time_point t0) {
   return std::chrono::duration<double, std::micro>(clk::now() - t0).count();
 }
 enum JobState { JOB_IDLE = 0, JOB_PENDING = 1, JOB_RUNNING = 2, JOB_DONE = 3 };
-enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_N };
+enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_N };
+constexpr int kEvRing = 16;   // forwards whose stage events may be outstanding
 }  // namespace
 
 struct feplb_ctx {
@@ -48,9 +49,16 @@ struct feplb_ctx {
 
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_counts = nullptr, ev_plan = nullptr;
-  cudaEvent_t ev[EV_N] = {nullptr};
+  cudaEvent_t evr[kEvRing][EV_N] = {{nullptr}};
+  cudaEvent_t* ev = evr[0];        // event set of the current forward
+  bool ev_used[kEvRing] = {false};
+  feplb_timeline ev_host[kEvRing]; // host fields of the forward that used the set
+  int ev_slot = 0;
   bool timeline_on = false, timeline_valid = false;
-  feplb_timeline tl;
+  feplb_timeline tl;               // host fields of the current forward
+  feplb_timeline tl_sum;           // totals over harvested forwards
+  feplb_timeline tl_last;          // last harvested forward
+  int64_t tl_n = 0;
   clk::time_point t0;
 
   // planner thread
@@ -204,7 +212,8 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaEventCreate(&c->ev_counts) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
-  for (int i = 0; ok && i < EV_N; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+  for (int r = 0; ok && r < kEvRing; ++r)
+    for (int i = 0; ok && i < EV_N; ++i) ok = cudaEventCreate(&c->evr[r][i]) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     feplb_destroy(c);
@@ -218,6 +227,8 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   c->plan = feplb_plan_out{0, 0, cap_moves, cap_groups, c->moves.data(), c->groups.data(),
                            c->load_before.data(), c->load_after.data()};
   memset(&c->tl, 0, sizeof(c->tl));
+  memset(&c->tl_sum, 0, sizeof(c->tl_sum));
+  memset(&c->tl_last, 0, sizeof(c->tl_last));
   c->th = std::thread(planner_main, c);
   *out = c;
   return FEPLB_OK;
@@ -248,8 +259,9 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->ev_counts) cudaEventDestroy(c->ev_counts);
   if (c->ev_plan) cudaEventDestroy(c->ev_plan);
-  for (int i = 0; i < EV_N; ++i)
-    if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+  for (int r = 0; r < kEvRing; ++r)
+    for (int i = 0; i < EV_N; ++i)
+      if (c->evr[r][i]) cudaEventDestroy(c->evr[r][i]);
   cudaGetLastError();
   delete c;
   return FEPLB_OK;
@@ -404,6 +416,32 @@ extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out*
   return FEPLB_OK;
 }
 
+// Reads the stage events of ring slot r (waiting for them if needed) and adds them to the totals.
+static int harvest_slot(feplb_ctx* c, int r) {
+  if (!c->ev_used[r]) return FEPLB_OK;
+  cudaEvent_t* ev = c->evr[r];
+  CUDA_TRY(c, cudaEventSynchronize(ev[EV_COMBINE]));
+  float ms = 0;
+  auto el = [&](cudaEvent_t a, cudaEvent_t b) { return cudaEventElapsedTime(&ms, a, b) == cudaSuccess ? ms * 1e3 : 0.0; };
+  feplb_timeline t = c->ev_host[r];
+  t.dev_hist_us = el(ev[EV_T0], ev[EV_HIST]);
+  t.dev_dispatch_us = el(ev[EV_HIST], ev[EV_DISPATCH]);
+  t.dev_static_ffn_us = el(ev[EV_STATIC0], ev[EV_STATIC1]);
+  t.dev_dynamic_ffn_us = el(ev[EV_DYN0], ev[EV_DYN1]);
+  t.dev_combine_us = el(ev[EV_DYN1], ev[EV_COMBINE]);
+  t.dev_counts_to_static_start_us = el(ev[EV_COUNTS], ev[EV_STATIC0]);
+  t.dev_counts_to_static_end_us = el(ev[EV_COUNTS], ev[EV_STATIC1]);
+  t.dev_total_us = el(ev[EV_T0], ev[EV_COMBINE]);
+  cudaGetLastError();
+  const double* src = reinterpret_cast<const double*>(&t);
+  double* dst = reinterpret_cast<double*>(&c->tl_sum);
+  for (size_t i = 0; i < sizeof(feplb_timeline) / sizeof(double); ++i) dst[i] += src[i];
+  c->tl_last = t;
+  c->tl_n += 1;
+  c->ev_used[r] = false;
+  return FEPLB_OK;
+}
+
 extern "C" int feplb_set_timeline(feplb_ctx* c, int32_t enable) {
   if (!c) return FEPLB_E_INVALID;
   c->timeline_on = enable != 0;
@@ -425,13 +463,19 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   const feplb_config& g = c->cfg;
   if (!dyn_mask_host && g.mask_policy != FEPLB_MASK_REACTIVE)
     return fail(c, FEPLB_E_INVALID, "moe_forward: dyn_mask_host is required unless mask_policy is REACTIVE");
+  int rc;
+  if (c->timeline_on) {
+    c->ev_slot = (c->ev_slot + 1) % kEvRing;
+    if ((rc = harvest_slot(c, c->ev_slot)) != FEPLB_OK) return rc;   // long finished unless the ring wrapped quickly
+    c->ev = c->evr[c->ev_slot];
+  }
   c->t0 = clk::now();
   c->timeline_valid = true;
-  int rc;
   TL_EVENT(EV_T0);
   // step 1: counts; the planner thread starts as soon as they reach the host
   if ((rc = feplb_route_hist(c, topk_ids, counts, rank_load, stream)) != FEPLB_OK) return rc;
   if ((rc = feplb_plan_async(c, counts, dyn_mask_host, stream)) != FEPLB_OK) return rc;
+  TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);
   // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move them here)
   rc = dispatch_impl(c, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, st);
@@ -466,6 +510,10 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   if ((rc = feplb_combine(c, y_perm, slot_to_row, gates, out, stream)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COMBINE);
   c->tl.host_return_us = us_since(c->t0);
+  if (c->timeline_on) {
+    c->ev_host[c->ev_slot] = c->tl;
+    c->ev_used[c->ev_slot] = true;
+  }
   return FEPLB_OK;
 }
 
@@ -497,23 +545,29 @@ extern "C" int feplb_moe_forward_host(feplb_ctx* c, const void* x_host, const in
 extern "C" int feplb_get_timeline(feplb_ctx* c, feplb_timeline* out) {
   if (!c || !out) return FEPLB_E_INVALID;
   if (!c->timeline_valid) return fail(c, FEPLB_E_STATE, "get_timeline: no forward pass yet");
-  feplb_timeline t = c->tl;
-  t.dev_hist_us = t.dev_dispatch_us = t.dev_static_ffn_us = t.dev_dynamic_ffn_us = t.dev_combine_us = 0;
-  t.dev_counts_to_static_start_us = t.dev_counts_to_static_end_us = t.dev_total_us = 0;
-  if (c->timeline_on) {
-    CUDA_TRY(c, cudaEventSynchronize(c->ev[EV_COMBINE]));
-    float ms = 0;
-    auto el = [&](cudaEvent_t a, cudaEvent_t b) { return cudaEventElapsedTime(&ms, a, b) == cudaSuccess ? ms * 1e3 : 0.0; };
-    t.dev_hist_us = el(c->ev[EV_T0], c->ev[EV_HIST]);
-    t.dev_dispatch_us = el(c->ev[EV_HIST], c->ev[EV_DISPATCH]);
-    t.dev_static_ffn_us = el(c->ev[EV_STATIC0], c->ev[EV_STATIC1]);
-    t.dev_dynamic_ffn_us = el(c->ev[EV_DYN0], c->ev[EV_DYN1]);
-    t.dev_combine_us = el(c->ev[EV_DYN1], c->ev[EV_COMBINE]);
-    t.dev_counts_to_static_start_us = el(c->ev_counts, c->ev[EV_STATIC0]);
-    t.dev_counts_to_static_end_us = el(c->ev_counts, c->ev[EV_STATIC1]);
-    t.dev_total_us = el(c->ev[EV_T0], c->ev[EV_COMBINE]);
-    cudaGetLastError();
+  if (c->timeline_on || c->tl_n) {
+    for (int i = 1; i <= kEvRing; ++i) {   // oldest first, so that tl_last is the newest forward
+      int rc = harvest_slot(c, (c->ev_slot + i) % kEvRing);
+      if (rc != FEPLB_OK) return rc;
+    }
+    *out = c->tl_last;
+  } else {
+    *out = c->tl;   // host fields only
   }
-  *out = t;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_timeline_totals(feplb_ctx* c, feplb_timeline* sum, int64_t* n_forwards, int32_t reset) {
+  if (!c || !sum || !n_forwards) return FEPLB_E_INVALID;
+  for (int i = 1; i <= kEvRing; ++i) {
+    int rc = harvest_slot(c, (c->ev_slot + i) % kEvRing);
+    if (rc != FEPLB_OK) return rc;
+  }
+  *sum = c->tl_sum;
+  *n_forwards = c->tl_n;
+  if (reset) {
+    memset(&c->tl_sum, 0, sizeof(c->tl_sum));
+    c->tl_n = 0;
+  }
   return FEPLB_OK;
 }

@@ -89,6 +89,7 @@ def lib() -> C.CDLL:
             "feplb_moe_forward_host": (C.c_int, [vp] * 20 + [C.POINTER(PlanOut), vp]),
             "feplb_set_timeline": (C.c_int, [vp, i32]),
             "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
+            "feplb_timeline_totals": (C.c_int, [vp, C.POINTER(Timeline), C.POINTER(i64), i32]),
             "feplb_launch_count": (i64, [vp]),
         }
         for name, (res, args) in sig.items():
@@ -287,6 +288,12 @@ class Context:
         t = Timeline()
         self._chk(lib().feplb_get_timeline(self._h, C.byref(t)), "feplb_get_timeline")
         return {n: getattr(t, n) for n, _ in Timeline._fields_}
+
+    def timeline_totals(self, reset=True):
+        """(sums over the timed forwards since the last reset, number of forwards)."""
+        t, n = Timeline(), C.c_int64()
+        self._chk(lib().feplb_timeline_totals(self._h, C.byref(t), C.byref(n), int(bool(reset))), "feplb_timeline_totals")
+        return {k: getattr(t, k) for k, _ in Timeline._fields_}, n.value
 
     def launch_count(self) -> int:
         return int(lib().feplb_launch_count(self._h))

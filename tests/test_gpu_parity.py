@@ -1,0 +1,383 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Integer results bit-exact; floating point within
+|gpu - ref| <= 1e-2 * max|ref| + 1e-2 * |ref| (bf16 inputs, fp32 accumulation)."""
+import numpy as np
+import pytest
+
+from oracle import feplb_oracle as O
+from paper_2604_19654_b200 import build as B
+from paper_2604_19654_b200 import feplb as F
+from paper_2604_19654_b200 import workloads as W
+
+from gpu_utils import DeviceCase, assert_close, oracle_mask, upload_groups
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    B.build()
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _tiny(T, K, E, R, d=128, f=64, **kw):
+    base = W.get_workload("cfg1")
+    return base.with_(name="tiny", T=T, K=K, E=E, R=R, d=d, f=f, **kw)
+
+
+# ----------------------------------------------------------------------------- integer stages
+
+HIST_CASES = [W.get_workload("cfg1"), W.get_workload("cfg2"), W.get_workload("cfg4"),
+              _tiny(1, 1, 4, 2), _tiny(37, 3, 6, 3), _tiny(1025, 5, 16, 4), _tiny(3000, 8, 128, 8),
+              _tiny(64, 2, 1, 1)]
+
+
+@pytest.mark.parametrize("w", HIST_CASES, ids=lambda w: f"{w.name}-T{w.T}K{w.K}E{w.E}")
+@pytest.mark.parametrize("A", [1, 128])
+def test_hist_and_dispatch_bit_exact(w, A):
+    torch = _torch()
+    ids, _ = W.gen_routing(w, 0) if w.E >= w.K and w.E > 1 else (np.zeros((w.T, w.K), np.int32), None)
+    if w.name == "tiny" and w.E >= 4:
+        rng = np.random.default_rng(w.T)
+        ids = rng.integers(0, w.E, size=(w.T, w.K)).astype(np.int32)      # duplicates inside a token are legal
+        ids[ids == 1] = 0                                                  # expert 1 stays empty
+    x = W.gen_activations(w, 0)
+    cfg = F.config_from_workload(w, row_align=A)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    d_ids, d_x = torch.from_numpy(ids).cuda(), F.bf16_tensor(x)
+    buf.x_perm.fill_(7.0)
+    ctx.route_hist(d_ids, buf.counts, buf.rank_load)
+    ctx.dispatch(d_x, d_ids, buf.counts, buf.x_perm, buf.slot_to_row, buf.row_to_token)
+    ctx.check_status()
+    counts, load = O.route_hist(ids, w.E, w.R)
+    s2r, r2t, pad_off, S_pad = O.permute(ids, w.E, A)
+    assert np.array_equal(buf.counts.cpu().numpy(), counts)
+    assert np.array_equal(buf.rank_load.cpu().numpy(), load)
+    assert np.array_equal(buf.slot_to_row.cpu().numpy()[: w.T], s2r)
+    g_r2t = buf.row_to_token.cpu().numpy()
+    assert np.array_equal(g_r2t[:S_pad], r2t)
+    assert np.all(g_r2t[S_pad:] == -1)
+    xp = O.gather_rows(x, r2t)
+    assert np.array_equal(F.bf16_bits(buf.x_perm)[:S_pad], xp)            # row copies and zero padding
+    ctx.close()
+
+
+def test_out_of_range_expert_id_is_reported_not_trapped():
+    torch = _torch()
+    w = _tiny(64, 2, 8, 2)
+    cfg = F.config_from_workload(w)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    ids = np.zeros((w.T, w.K), np.int32)
+    ids[5, 1] = 8
+    ids[9, 0] = -3
+    ctx.route_hist(torch.from_numpy(ids).cuda(), buf.counts, buf.rank_load)
+    with pytest.raises(F.FeplbError) as ei:
+        ctx.check_status()
+    assert ei.value.code == F.E_RANGE
+    assert int(buf.counts.sum()) == w.T * w.K - 2
+    ctx.check_status()                                                    # the status word was cleared
+    ctx.close()
+
+
+def test_dispatch_with_wrong_counts_is_reported():
+    torch = _torch()
+    w = _tiny(64, 2, 8, 2)
+    cfg = F.config_from_workload(w)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    ids = np.random.default_rng(0).integers(0, 8, size=(w.T, w.K)).astype(np.int32)
+    d_ids = torch.from_numpy(ids).cuda()
+    ctx.route_hist(d_ids, buf.counts, buf.rank_load)
+    buf.counts[3] += 1
+    ctx.dispatch(F.bf16_tensor(W.gen_activations(w, 0)), d_ids, buf.counts, buf.x_perm, buf.slot_to_row, buf.row_to_token)
+    with pytest.raises(F.FeplbError) as ei:
+        ctx.check_status()
+    assert ei.value.code == F.E_DEVICE
+    ctx.close()
+
+
+def test_home_groups_match_the_no_move_plan():
+    torch = _torch()
+    for w, A in ((W.get_workload("cfg2"), 1), (W.get_workload("cfg1"), 128)):
+        ids, _ = W.gen_routing(w, 1)
+        cfg = F.config_from_workload(w, row_align=A)
+        ctx, buf = F.Context(cfg), F.Buffers(cfg)
+        ctx.route_hist(torch.from_numpy(ids).cuda(), buf.counts, buf.rank_load)
+        groups = torch.zeros(w.E, 5, dtype=torch.int32, device="cuda")
+        mask_out = torch.zeros(w.E, dtype=torch.uint8, device="cuda")
+        ctx.home_groups(buf.counts, None, groups, mask_out)               # REACTIVE: mask from counts on the device
+        counts, _ = O.route_hist(ids, w.E, w.R)
+        mask = oracle_mask(counts, w)
+        assert np.array_equal(mask_out.cpu().numpy(), mask)
+        pad_off, _ = O.segment_offsets(counts, A)
+        exp = [(e, int(pad_off[e]), int(counts[e]), e // w.L, int(mask[e])) for e in range(w.E)]
+        assert [tuple(r) for r in groups.cpu().numpy().tolist()] == exp
+        # the oracle's plan with an empty mask lists the same non-empty groups
+        p = O.plan(counts, np.zeros(w.E, np.uint8), w.R, row_align=A)
+        assert [g[:4] for g in p["groups"]] == [g[:4] for g in exp if g[2] > 0]
+        ctx.close()
+
+
+# ----------------------------------------------------------------------------- expert FFN
+
+def _ffn_case(E, d, f, rows_per_expert, A=1, seed=0, order=None):
+    """Builds x_perm / groups for the given per-expert row counts and checks H-free Y parity."""
+    torch = _torch()
+    rng = np.random.default_rng(seed)
+    counts = np.asarray(rows_per_expert)
+    pad_off, S_pad = O.segment_offsets(counts, A)
+    w = _tiny(max(int(counts.sum()), 1), 1, E, 1, d=d, f=f)
+    cfg = F.config_from_workload(w, row_align=A)
+    ctx = F.Context(cfg)
+    cap = F.s_pad(cfg)
+    xb = W.f32_to_bf16_bits((rng.standard_normal((cap, d)) * 0.5).astype(np.float32))
+    w1 = W.f32_to_bf16_bits((rng.standard_normal((E, f, d)) / np.sqrt(d)).astype(np.float32))
+    w3 = W.f32_to_bf16_bits((rng.standard_normal((E, f, d)) / np.sqrt(d)).astype(np.float32))
+    w2 = W.f32_to_bf16_bits((rng.standard_normal((E, d, f)) / np.sqrt(f)).astype(np.float32))
+    row_expert = np.full(cap, -1, np.int64)
+    groups = []
+    for e in range(E):
+        row_expert[pad_off[e]: pad_off[e] + counts[e]] = e
+        groups.append((e, int(pad_off[e]), int(counts[e]), 0, e % 2))
+    if order is not None:
+        groups = [groups[i] for i in order]
+    d_x, d_w1, d_w3, d_w2 = (F.bf16_tensor(a) for a in (xb, w1, w3, w2))
+    h = torch.zeros(cap, f, dtype=torch.bfloat16, device="cuda")
+    y = torch.full((cap, d), 3.0, dtype=torch.bfloat16, device="cuda")
+    d_groups = upload_groups(groups)
+    ctx.expert_ffn(d_x, d_w1, d_w3, d_w2, d_groups, len(groups), h, y, which=F.FFN_STATIC)
+    ctx.expert_ffn(d_x, d_w1, d_w3, d_w2, d_groups, len(groups), h, y, which=F.FFN_DYNAMIC)
+    ctx.check_status()
+    ref = O.expert_ffn(xb, row_expert, w1, w3, w2)
+    got = W.bf16_bits_to_f64(F.bf16_bits(y))
+    live = row_expert >= 0
+    worst = assert_close(got[live], ref[live], f"FFN E={E} d={d} f={f}")
+    assert np.all(got[~live] == 3.0)                                      # rows outside the groups are untouched
+    ctx.close()
+    return worst
+
+
+@pytest.mark.parametrize("E,d,f,rows", [
+    (1, 128, 64, [128]),                       # one full tile, smallest shapes (bn = 64 in both passes)
+    (1, 128, 64, [1]),                         # a single row
+    (2, 128, 64, [5, 200]),                    # ragged last tiles
+    (4, 256, 128, [0, 129, 0, 383]),           # empty experts; bn = 128 in both passes
+    (3, 512, 192, [300, 17, 128]),             # f % 128 != 0 -> bn = 64 in pass 1, 128 in pass 2
+    (8, 384, 256, [64, 1, 0, 257, 128, 127, 513, 2]),   # d % 256 != 0 -> bn = 64 in pass 2
+    (2, 2048, 768, [700, 45]),                 # the mid layer's shapes: 32 K blocks wrap the 4-stage ring
+])
+def test_expert_ffn_parity(E, d, f, rows):
+    _ffn_case(E, d, f, rows)
+
+
+def test_expert_ffn_padded_segments_and_group_order():
+    _ffn_case(5, 256, 128, [130, 0, 7, 256, 90], A=128)
+    _ffn_case(5, 256, 128, [130, 0, 7, 256, 90], A=1, order=[4, 2, 0, 3, 1])
+
+
+def test_expert_ffn_many_tiles_per_cta():
+    # more tiles than CTAs: every CTA walks several tiles, both accumulator stages and phases flip
+    _ffn_case(6, 256, 128, [4000, 3000, 2500, 1, 6000, 777])
+
+
+def test_expert_ffn_rejects_bad_group_without_trapping():
+    torch = _torch()
+    w = _tiny(128, 1, 2, 1)
+    cfg = F.config_from_workload(w)
+    ctx = F.Context(cfg)
+    cap = F.s_pad(cfg)
+    z = torch.zeros(cap, 128, dtype=torch.bfloat16, device="cuda")
+    wz = torch.zeros(2, 64, 128, dtype=torch.bfloat16, device="cuda")
+    w2z = torch.zeros(2, 128, 64, dtype=torch.bfloat16, device="cuda")
+    h = torch.zeros(cap, 64, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(cap, 128, dtype=torch.bfloat16, device="cuda")
+    bad = upload_groups([(5, 0, 10, 0, 0), (0, 100, 100, 0, 0)])          # expert out of range; rows past the buffer
+    ctx.expert_ffn(z, wz, wz, w2z, bad, 2, h, y)
+    with pytest.raises(F.FeplbError) as ei:
+        ctx.check_status()
+    assert ei.value.code == F.E_DEVICE
+    with pytest.raises(F.FeplbError):
+        ctx.expert_ffn(z, wz, wz, w2z, bad, 5000, h, y)                   # more groups than the table holds
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- combine
+
+@pytest.mark.parametrize("T,K,d", [(1, 1, 128), (33, 2, 128), (257, 6, 2048), (100, 8, 6144), (50, 32, 256)])
+def test_combine_parity(T, K, d):
+    torch = _torch()
+    rng = np.random.default_rng(T * K)
+    w = _tiny(T, K, 32, 1, d=d)
+    cfg = F.config_from_workload(w)
+    ctx = F.Context(cfg)
+    rows = T * K
+    y = W.f32_to_bf16_bits(rng.standard_normal((rows, d)).astype(np.float32))
+    s2r = rng.permutation(rows).astype(np.int32).reshape(T, K)
+    gates = rng.random((T, K)).astype(np.float32)
+    out = torch.zeros(T, d, dtype=torch.bfloat16, device="cuda")
+    ctx.combine(F.bf16_tensor(y), torch.from_numpy(s2r).cuda(), torch.from_numpy(gates).cuda(), out)
+    ref = O.combine(W.bf16_bits_to_f64(y), s2r, gates)
+    got = W.bf16_bits_to_f64(F.bf16_bits(out))
+    # one bf16 rounding of the result (2^-9 relative) plus fp32 accumulation error on the sum of |terms|
+    mag = O.combine(np.abs(W.bf16_bits_to_f64(y)), s2r, gates)
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -20 * mag + 1e-30)
+    ctx.close()
+
+
+def test_dispatch_then_combine_is_the_identity_for_k1():
+    torch = _torch()
+    w = _tiny(777, 1, 16, 4, d=256)
+    cfg = F.config_from_workload(w, row_align=128)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    ids = np.random.default_rng(1).integers(0, 16, size=(w.T, 1)).astype(np.int32)
+    x = W.gen_activations(w, 0)
+    d_ids = torch.from_numpy(ids).cuda()
+    ctx.route_hist(d_ids, buf.counts, buf.rank_load)
+    ctx.dispatch(F.bf16_tensor(x), d_ids, buf.counts, buf.x_perm, buf.slot_to_row, buf.row_to_token)
+    ctx.combine(buf.x_perm, buf.slot_to_row, torch.ones(w.T, 1, device="cuda"), buf.out)
+    ctx.check_status()
+    assert np.array_equal(F.bf16_bits(buf.out)[: w.T], x)
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- whole layer
+
+def _check_forward(case, split=0, sample=None):
+    w = case.w
+    p = case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    case.ctx.check_status()
+    counts, load = O.route_hist(case.ids, w.E, w.R)
+    mask = oracle_mask(counts, w)
+    A = case.cfg.row_align
+    op = O.plan(counts, mask, w.R, tau=case.cfg.tau, max_num_dyn=case.cfg.max_num_dyn, policy=case.cfg.policy,
+                split=case.cfg.split, split_granule=case.cfg.split_granule, row_align=A)
+    # integer outputs bit-exact: counts, per-rank loads before/after, moves, groups, permutation
+    assert np.array_equal(case.buf.counts.cpu().numpy(), counts)
+    assert np.array_equal(case.buf.rank_load.cpu().numpy(), load)
+    assert p.moves == [tuple(int(v) for v in m) for m in op["moves"]]
+    assert p.groups == [tuple(int(v) for v in g) for g in op["groups"]]
+    assert np.array_equal(p.load_before, op["load_before"]) and np.array_equal(p.load_after, op["load_after"])
+    s2r, r2t, _, S_pad = O.permute(case.ids, w.E, A)
+    assert np.array_equal(case.buf.slot_to_row.cpu().numpy()[: w.T], s2r)
+    assert np.array_equal(case.buf.row_to_token.cpu().numpy()[:S_pad], r2t)
+    assert O.straggler_ratio(op["load_after"]) <= O.straggler_ratio(op["load_before"])
+    got = W.bf16_bits_to_f64(F.bf16_bits(case.buf.out))[: w.T]
+    tokens = None if sample is None else np.sort(np.random.default_rng(5).choice(w.T, size=sample, replace=False))
+    ref = O.moe_layer(case.x, case.ids, case.gates, case.w1, case.w3, case.w2, w.E, tokens=tokens)
+    assert_close(got if tokens is None else got[tokens], ref, f"layer output {w.name}")
+    return p, op
+
+
+@pytest.mark.parametrize("A", [1, 128])
+def test_forward_cfg1(A):
+    case = DeviceCase(W.get_workload("cfg1"), row_align=A)
+    p, _ = _check_forward(case)
+    assert len(p.moves) >= 1
+    # a second pass on the same context gives bit-identical results (determinism)
+    out1 = F.bf16_bits(case.buf.out).copy()
+    y1 = F.bf16_bits(case.buf.y_perm).copy()
+    case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    _torch().cuda.synchronize()
+    assert np.array_equal(F.bf16_bits(case.buf.out), out1)
+    n_live = int(case.ids.size)
+    assert np.array_equal(F.bf16_bits(case.buf.y_perm)[:n_live], y1[:n_live]) or A == 128
+    case.close()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_forward_cfg1_other_seeds(seed):
+    w = W.get_workload("cfg1")
+    case = DeviceCase(w, mb=10 + seed)
+    _check_forward(case)
+    case.close()
+
+
+def test_forward_cfg2_full():
+    w = W.get_workload("cfg2")
+    weights = W.gen_weights(w)
+    for mb in (0, 3):
+        case = DeviceCase(w, mb=mb, weights=weights)
+        _check_forward(case, sample=None if mb == 0 else 256)
+        case.close()
+
+
+@pytest.mark.parametrize("split", [0, 1])
+def test_forward_cfg4_extreme_skew(split):
+    w = W.get_workload("cfg4")
+    case = DeviceCase(w, mb=0, split=split)
+    p, op = _check_forward(case, sample=512)
+    if split:
+        assert any(rows < max(c, 1) for (e, _, _, rows) in p.moves
+                   for c in [int(np.bincount(case.ids.ravel(), minlength=w.E)[e])])   # a hot expert was cut
+    case.close()
+
+
+def test_forward_given_mask_and_literal_policy():
+    w = W.get_workload("cfg2").with_(T=512)
+    mask = np.zeros(w.E, np.uint8)
+    mask[::4] = 1
+    case = DeviceCase(w, mb=2, mask_policy=F.MASK_GIVEN, policy=F.POLICY_LITERAL)
+    p = case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf,
+                             dyn_mask_host=mask)
+    case.ctx.check_status()
+    counts, _ = O.route_hist(case.ids, w.E, w.R)
+    op = O.plan(counts, mask, w.R, tau=w.tau, max_num_dyn=w.max_num_dyn, policy=O.POLICY_LITERAL)
+    assert p.moves == [tuple(int(v) for v in m) for m in op["moves"]]
+    assert p.groups == [tuple(int(v) for v in g) for g in op["groups"]]
+    got = W.bf16_bits_to_f64(F.bf16_bits(case.buf.out))[: w.T]
+    ref = O.moe_layer(case.x, case.ids, case.gates, case.w1, case.w3, case.w2, w.E)
+    assert_close(got, ref, "layer output, given mask")
+    with pytest.raises(F.FeplbError):                                      # a mask is mandatory in this mode
+        case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    case.close()
+
+
+def test_forward_host_buffers_and_timeline():
+    torch = _torch()
+    w = W.get_workload("cfg1")
+    case = DeviceCase(w)
+    case.ctx.set_timeline(True)
+    xh = torch.from_numpy(case.x.view(np.int16)).pin_memory()
+    ih = torch.from_numpy(case.ids).pin_memory()
+    gh = torch.from_numpy(case.gates).pin_memory()
+    oh = torch.zeros(w.T, w.d, dtype=torch.int16).pin_memory()
+    x_dev = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
+    i_dev = torch.empty(w.T, w.K, dtype=torch.int32, device="cuda")
+    g_dev = torch.empty(w.T, w.K, dtype=torch.float32, device="cuda")
+    case.ctx.moe_forward_host(xh, ih, gh, x_dev, i_dev, g_dev, case.d_w1, case.d_w3, case.d_w2, case.buf, oh)
+    case.ctx.check_status()
+    ref = O.moe_layer(case.x, case.ids, case.gates, case.w1, case.w3, case.w2, w.E)
+    assert_close(W.bf16_bits_to_f64(oh.numpy().view(np.uint16)), ref, "host-buffer forward")
+    tl = case.ctx.get_timeline()
+    assert tl["dev_total_us"] > 0 and tl["host_plan_done_us"] >= tl["host_counts_ready_us"] > 0
+    assert tl["dev_static_ffn_us"] > 0 and tl["plan_us"] >= 0
+    assert case.ctx.launch_count() > 0
+    case.close()
+
+
+def test_plan_wait_without_request_and_timeout_paths():
+    w = W.get_workload("cfg1")
+    cfg = F.config_from_workload(w)
+    ctx = F.Context(cfg)
+    with pytest.raises(F.FeplbError) as ei:
+        ctx.plan_wait(10)
+    assert ei.value.code == F.E_STATE
+    ctx.close()
+
+
+def test_empty_batch():
+    w = _tiny(0, 2, 8, 2)
+    cfg = F.config_from_workload(w)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    torch = _torch()
+    z = torch.zeros(1, 128, dtype=torch.bfloat16, device="cuda")
+    zi = torch.zeros(1, 2, dtype=torch.int32, device="cuda")
+    wz = torch.zeros(8, 64, 128, dtype=torch.bfloat16, device="cuda")
+    w2z = torch.zeros(8, 128, 64, dtype=torch.bfloat16, device="cuda")
+    p = ctx.moe_forward(z, zi, torch.zeros(1, 2, device="cuda"), wz, wz, w2z, buf)
+    ctx.check_status()
+    assert p.moves == [] and p.groups == [] and int(buf.counts.sum()) == 0
+    ctx.close()
