@@ -57,7 +57,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(self.gpu)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -167,6 +167,28 @@ def _config_dict(w, args, extra=None):
     return c
 
 
+# --------------------------------------------------------------------------------------------- sharding
+
+def rank_microbatches(rank, n_mb):
+    """Micro-batch seeds of one rank: every rank owns its own, disjoint, block (weak scaling)."""
+    return [rank * n_mb + i for i in range(n_mb)]
+
+
+def max_over_ranks(ms, world, device):
+    """Slowest rank's time; an all-reduce(MAX) when there is more than one rank."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(world, steps, tokens_per_step, ms):
+    """Tokens all ranks processed over the slowest rank's time."""
+    return world * steps * tokens_per_step / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------------------------- CUDA arm
 
 def gemm_flops(w):
@@ -196,7 +218,7 @@ def run_cuda(args, w):
     weights = W.gen_weights(w)
     d_w1, d_w3, d_w2 = (F.bf16_tensor(a) for a in weights)
     n_mb = w.n_microbatches
-    host = [W.gen_microbatch(w, rank * n_mb + i) for i in range(n_mb)]      # every rank its own micro-batches
+    host = [W.gen_microbatch(w, mb) for mb in rank_microbatches(rank, n_mb)]
     dev = [(F.bf16_tensor(x), torch.from_numpy(i).cuda(), torch.from_numpy(g).cuda()) for x, i, g in host]
     stream = torch.cuda.current_stream()
 
@@ -233,13 +255,27 @@ def run_cuda(args, w):
     totals, n_fw = ctx.timeline_totals(reset=True)
     ctx.set_timeline(False)
     ctx.check_status()
-    t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    value = world * args.steps * w.T / (ms_total * 1e-3)
+    ms_total = max_over_ranks(ms_total, world, "cuda")
+    value = whole_job_throughput(world, args.steps, w.T, ms_total)
 
     # ---- end to end through the host-buffer entry point -----------------------------------------
+    e2e_value, h2d, d2h = None, w.T * w.d * 2 + 2 * w.T * w.K * 4, w.T * w.d * 2
+    if not args.quick:
+        e2e_value = _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world, n_mb)
+
+    # ---- stragglers: token loads from the plan; GEMM time of every virtual rank run alone ---------
+    strag = None
+    if rank == 0 and not args.no_straggler and not args.quick:
+        strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb)
+    _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals, n_fw, e2e_value, h2d, d2h, strag, weights, n_mb)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world, n_mb):
+    import torch
+    import torch.distributed as dist
     pinned = []
     for x, i, g in host:
         pinned.append((torch.from_numpy(x.view(np.int16)).pin_memory(), torch.from_numpy(i).pin_memory(),
@@ -265,18 +301,10 @@ def run_cuda(args, w):
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), 0.0)
     del t0
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * args.steps * w.T / (float(t.item()) * 1e-3)
-    h2d = w.T * w.d * 2 + 2 * w.T * w.K * 4
-    d2h = w.T * w.d * 2
+    return whole_job_throughput(world, args.steps, w.T, max_over_ranks(e2e_ms, world, "cuda"))
 
-    # ---- stragglers: token loads from the plan; GEMM time of every virtual rank run alone ---------
-    strag = None
-    if rank == 0 and not args.no_straggler:
-        strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb)
 
+def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals, n_fw, e2e_value, h2d, d2h, strag, weights, n_mb):
     if rank == 0:
         peaks = _peaks()
         ffn_us = totals["dev_static_ffn_us"] + totals["dev_dynamic_ffn_us"]
@@ -296,21 +324,20 @@ def run_cuda(args, w):
                 "hbm_peak_gbs": peaks["hbm_gbs"]}
         stage_us = {k: (v / n_fw if n_fw else None) for k, v in totals.items()}
         # CPU oracle on the host cores: a bounded sample of the same workload
-        cpu_val, cpu_ms, n_tok = time_oracle(w, 2, 1, min(w.T, 4096), weights)
+        cpu = None
+        if not args.quick:
+            cpu_val, cpu_ms, n_tok = time_oracle(w, 2, 1, min(w.T, 4096), weights)
+            cpu = {"value": cpu_val, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
+                   "sample": f"first {n_tok} tokens of 2 micro-batches, whole path (numpy fp64 oracle)"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": _config_dict(w, args),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
-            "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
-                             "sample": f"first {n_tok} tokens of 2 micro-batches, whole path (numpy fp64 oracle)"},
-            "stage_us": stage_us, "straggler": strag,
+            "cpu_baseline": cpu, "stage_us": stage_us, "straggler": strag,
         }
         print(json.dumps(line), flush=True)
-    ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
 
 
 def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb, reps=3):
@@ -358,12 +385,14 @@ def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb,
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-sample-tokens", type=int, default=1024)
     ap.add_argument("--no-straggler", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     args = ap.parse_args()
     w = W.get_workload(args.workload)
     if args.impl == "reference":
