@@ -166,6 +166,30 @@ int feplb_route_hist(feplb_ctx* ctx, const int32_t* topk_ids, int32_t* counts, i
 int feplb_dispatch(feplb_ctx* ctx, const void* x, const int32_t* topk_ids, const int32_t* counts,
                    void* x_perm, int32_t* slot_to_row, int32_t* row_to_token, void* stream);
 
+/* Largest ceil(T*K/1024) * E that feplb_dispatch_noalloc accepts (ints of built-in scratch). */
+#define FEPLB_NOALLOC_MAX_HIST_INTS 524288
+
+/* (The paper has no counterpart to this entry point; it exists for deployment reasons only.)
+ * feplb_dispatch for callers that cannot allocate device memory where they need a dispatch --
+ * e.g. a server whose own pool already owns all free device memory, or a loop that cannot take
+ * the device-wide synchronisation of cudaMalloc/cudaFree -- and therefore cannot create a
+ * context either.  Same inputs, outputs and results as feplb_dispatch (cfg replaces the
+ * context); the permutation's scratch is a ~2 MiB array built into the library image, resident
+ * on every GPU that loads the library until the process exits.  This call allocates and frees
+ * nothing, on the device or through any library.
+ *   - Limit: ceil(T*K/1024) * E <= FEPLB_NOALLOC_MAX_HIST_INTS, else FEPLB_E_NOMEM is returned
+ *     and nothing is enqueued (use feplb_dispatch).
+ *   - The first call on each device looks the array's device address up once (with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the array, which keeps the previous call's contents (the
+ *     kernels overwrite what they read before reading it).  Calls whose GPU work overlaps --
+ *     other streams or threads -- race on it: serialise them.
+ *   - status: dev uint32, zeroed by the caller, receives error bits (1 = expert id out of range,
+ *     2 = counts disagree with topk_ids); NULL to ignore them. */
+int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, const int32_t* topk_ids,
+                           const int32_t* counts, void* x_perm, int32_t* slot_to_row,
+                           int32_t* row_to_token, uint32_t* status, void* stream);
+
 /* Writes the E-entry group table {e, pad_off[e], counts[e], home(e), dyn_mask[e]} to
  * groups_out (dev), from device-resident counts and mask, without involving the host: the
  * table the static-expert GEMM runs on while the planner works (Section 2.3 timeline).

@@ -13,7 +13,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfeplb.so")
-SOURCES = ["feplb_plan.cpp", "feplb_api.cu", "feplb_route.cu", "feplb_combine.cu", "feplb_gemm.cu"]
+SOURCES = ["feplb_plan.cpp", "feplb_api.cu", "feplb_route.cu", "feplb_combine.cu", "feplb_gemm.cu",
+           "feplb_noalloc.cu"]
 
 
 def _nvcc() -> str:

@@ -11,6 +11,9 @@
 #define FEPLB_MAX_GROUPS 1024
 #define FEPLB_SLOTS_PER_BLOCK 1024   // slots ranked by one CTA of the permutation kernels
 #define FEPLB_TILE_M 128             // rows of one GEMM tile
+#ifndef FEPLB_NOALLOC_MAX_HIST_INTS
+#error "feplb.h must define FEPLB_NOALLOC_MAX_HIST_INTS"
+#endif
 
 // bits of the device status word
 #define FEPLB_ST_RANGE 1u      // expert id outside [0, E)

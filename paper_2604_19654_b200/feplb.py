@@ -80,6 +80,7 @@ def lib() -> C.CDLL:
             "feplb_plan": (C.c_int, [C.POINTER(Config), C.POINTER(i32), C.POINTER(C.c_uint8), C.POINTER(PlanOut)]),
             "feplb_route_hist": (C.c_int, [vp, vp, vp, vp, vp]),
             "feplb_dispatch": (C.c_int, [vp] * 8),
+            "feplb_dispatch_noalloc": (C.c_int, [C.POINTER(Config)] + [vp] * 8),
             "feplb_home_groups": (C.c_int, [vp] * 6),
             "feplb_expert_ffn": (C.c_int, [vp, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]),
             "feplb_combine": (C.c_int, [vp] * 6),
@@ -167,6 +168,19 @@ def plan(cfg: Config, counts, dyn_mask) -> Plan:
     if rc:
         raise FeplbError(rc, "feplb_plan")
     return p
+
+
+def dispatch_noalloc(cfg: Config, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, status=None, stream=None):
+    """Dispatch without a context and without any allocation (scratch is built into the library).
+
+    For callers that cannot allocate device memory at this point (their own pool owns it all, or
+    they cannot take cudaMalloc's synchronisation).  Same results as ``Context.dispatch``.  Calls
+    on one device must not overlap on the GPU; sizes beyond the built-in scratch raise E_NOMEM.
+    """
+    rc = lib().feplb_dispatch_noalloc(C.byref(cfg), _ptr(x), _ptr(topk_ids), _ptr(counts), _ptr(x_perm),
+                                      _ptr(slot_to_row), _ptr(row_to_token), _ptr(status), Context._stream(stream))
+    if rc:
+        raise FeplbError(rc, "feplb_dispatch_noalloc")
 
 
 def _ptr(t) -> Optional[int]:
