@@ -40,6 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC,-pthread",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    cmd[1:1] = os.environ.get("FEPLB_NVCC_FLAGS", "").split()      # e.g. -DFEPLB_GEMM_BK=32 for experiments
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     r = subprocess.run(cmd, capture_output=True, text=True)

@@ -7,6 +7,7 @@
 #include <condition_variable>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -472,25 +473,38 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   c->t0 = clk::now();
   c->timeline_valid = true;
   TL_EVENT(EV_T0);
-  // step 1: counts; the planner thread starts as soon as they reach the host
-  if ((rc = feplb_route_hist(c, topk_ids, counts, rank_load, stream)) != FEPLB_OK) return rc;
+  // step 1: counts, rank loads, segment offsets and the home group table in two launches; the
+  // planner thread starts as soon as the counts reach the host
+  if (!counts || !rank_load || !row_to_token) return fail(c, FEPLB_E_INVALID, "moe_forward: null pointer");
+  if (g.T > 0) {
+    if ((rc = check_dev_ptrs(c, {x, x_perm})) != FEPLB_OK) return rc;
+    if (!topk_ids || !slot_to_row) return fail(c, FEPLB_E_INVALID, "moe_forward: null pointer");
+  }
+  const int64_t S = (int64_t)g.T * g.K;
+  const uint8_t* mask_dev = nullptr;
+  if (dyn_mask_host) {
+    memcpy(c->h_mask, dyn_mask_host, g.E);
+    CUDA_TRY(c, cudaMemcpyAsync(c->d_mask, c->h_mask, g.E, cudaMemcpyHostToDevice, st));
+    mask_dev = c->d_mask;
+  }
+  CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
+                                       rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
+                                       (int64_t)c->s_cap, c->d_status, st, &c->launches));
   if ((rc = feplb_plan_async(c, counts, dyn_mask_host, stream)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);
-  // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move them here)
-  rc = dispatch_impl(c, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, st);
-  TL_EVENT(EV_DISPATCH);
-  // step 4: static experts on their home ranks, from a group table built on the device
-  if (rc == FEPLB_OK) {
-    const uint8_t* mask_dev = nullptr;
-    if (dyn_mask_host) {
-      memcpy(c->h_mask, dyn_mask_host, g.E);
-      cudaError_t e = cudaMemcpyAsync(c->d_mask, c->h_mask, g.E, cudaMemcpyHostToDevice, st);
-      if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "mask upload: %s", cudaGetErrorString(e));
-      mask_dev = c->d_mask;
-    }
-    if (rc == FEPLB_OK) rc = feplb_home_groups(c, counts, mask_dev, c->d_home_groups, nullptr, stream);
+  // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move
+  // them here).  From here on a failure must still join the planner, so errors are carried in rc.
+  {
+    cudaError_t e = feplb_launch_rank(topk_ids, S, g.K, g.E, c->d_block_hist, c->d_pad_off, slot_to_row, row_to_token,
+                                      (int64_t)c->s_cap, st, &c->launches);
+    if (e == cudaSuccess)
+      e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align, st,
+                              &c->launches, row_to_token);
+    if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "dispatch launch: %s", cudaGetErrorString(e));
   }
+  TL_EVENT(EV_DISPATCH);
+  // step 4: static experts on their home ranks, from the group table built on the device
   TL_EVENT(EV_STATIC0);
   if (rc == FEPLB_OK)
     rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st);

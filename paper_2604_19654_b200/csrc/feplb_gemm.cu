@@ -7,11 +7,10 @@
 //                    the two halves of the accumulator and rounds to bf16
 //   pass 2 (plain):  Y[rows, n0:n0+2bn] = H W2[e]
 // Per CTA: warp 0 = TMA producer (one lane), warp 1 = tcgen05.mma issuer (one lane) and TMEM
-// owner, warps 2..5 = epilogue (tcgen05.ld -> registers -> global).  A and B tiles are staged
-// by TMA (128-byte swizzle, K-major) through a 4-stage shared-memory ring; the fp32 accumulator
-// lives in TMEM and is double-buffered so the epilogue of tile i overlaps the MMAs of tile
-// i+1.  A tile is 128 rows of ONE group (row segment of one expert); the last tile of a group
-// is ragged and its surplus rows are computed but never stored.
+// owner, the other warps = epilogue (tcgen05.ld -> registers -> global).  A and B tiles are
+// staged by TMA (128-byte swizzle, K-major) through a shared-memory ring; the fp32 accumulators
+// live in TMEM.  A tile covers rows of ONE group (row segment of one expert); the last tile of
+// a group is ragged and its surplus rows are computed but never stored.
 //
 // Every mbarrier wait is bounded: when it gives up the CTA raises FEPLB_ST_WAIT in the status
 // word, all roles leave their loops, TMEM is released and the kernel returns.
@@ -25,18 +24,23 @@
 
 namespace {
 
-constexpr int BM = FEPLB_TILE_M;       // rows per tile (UMMA M)
+constexpr int BM = FEPLB_TILE_M;       // rows per MMA (UMMA M) = rows of one sub-tile
 constexpr int BK = 64;                 // K elements per stage = one 128-byte swizzle row
 constexpr int UMMA_K = 16;             // K per tcgen05.mma for 16-bit inputs
+constexpr int kAccCols = 256;          // TMEM columns of one accumulator
+constexpr int kTmemCols = 512;         // all of TMEM: one CTA per SM
+constexpr int kABytes = BM * BK * 2;               // 16 KiB per sub-tile
+constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
+constexpr unsigned long long kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s per wait
+
+// Tile 128 x 256 (UMMA M x N), K step 64: 4 stages of 48 KiB (A 16 KiB + B 32 KiB); two
+// accumulators in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1.
 constexpr int kStages = 4;
 constexpr int kAccStages = 2;
-constexpr int kAccCols = 256;          // TMEM columns per accumulator stage
-constexpr int kTmemCols = kAccStages * kAccCols;   // 512 = all of TMEM: one CTA per SM
-constexpr int kThreads = 192;
-constexpr int kABytes = BM * BK * 2;               // 16 KiB
-constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytesMax;  // 48 KiB, a multiple of 1024
-constexpr unsigned long long kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s per wait
+constexpr int kStageBytes = kABytes + kBBytesMax;   // 48 KiB, a multiple of 1024
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kEpiStageBytes = 32 * 128;            // per epilogue warp: 32 rows x 64 bf16
 
 struct SmemTail {
   unsigned long long full[kStages];
@@ -45,12 +49,13 @@ struct SmemTail {
   unsigned long long tmem_empty[kAccStages];
   uint32_t tmem_base;
   int abort_flag;
-  int prefix[FEPLB_MAX_GROUPS + 1];   // prefix[g] = M-tiles of groups before g
+  int prefix[FEPLB_MAX_GROUPS + 1];   // prefix[g] = M tiles of groups before g
   int g_row_start[FEPLB_MAX_GROUPS];
   int g_rows[FEPLB_MAX_GROUPS];
   int g_expert[FEPLB_MAX_GROUPS];
 };
-constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes + sizeof(SmemTail);
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes +
+                              (size_t)kEpiWarps * kEpiStageBytes + sizeof(SmemTail);
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 static_assert(kSmemBytes > 116 * 1024, "two CTAs must never share an SM: each allocates all of TMEM");
 
@@ -64,7 +69,6 @@ struct GemmParams {
   int num_k_blocks;     // K / 64
   int b_rows_per_expert;  // rows of one expert in the B tensor maps
   int bn;               // rows of one B half tile (64 or 128); the MMA has N = 2*bn
-  int swiglu;           // 1: out = silu(acc[:bn]) * acc[bn:], bn columns; 0: out = acc, 2*bn columns
   __nv_bfloat16* out;
   int ld_out;           // elements between output rows
   uint32_t* status;
@@ -209,12 +213,28 @@ __device__ __forceinline__ TileCoord tile_coord(const SmemTail* t, int n_groups,
   return c;
 }
 
+// fp32 accumulator registers of 32 columns -> 16 packed bf16 pairs (SwiGLU: silu(a) * b first).
+template <bool SWIGLU>
+__device__ __forceinline__ void convert_slice(const uint32_t (&a)[32], const uint32_t (&b)[32], uint32_t* packed) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float v0 = __uint_as_float(a[2 * i]), v1 = __uint_as_float(a[2 * i + 1]);
+    if (SWIGLU) {
+      v0 = silu_f(v0) * __uint_as_float(b[2 * i]);
+      v1 = silu_f(v1) * __uint_as_float(b[2 * i + 1]);
+    }
+    packed[i] = pack_bf16x2(v0, v1);
+  }
+}
+
+template <bool SWIGLU>
 __global__ void __launch_bounds__(kThreads, 1)
 k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  SmemTail* tail = reinterpret_cast<SmemTail*>(smem + (size_t)kStages * kStageBytes);
+  uint8_t* epi_smem = smem + (size_t)kStages * kStageBytes;
+  SmemTail* tail = reinterpret_cast<SmemTail*>(epi_smem + (size_t)kEpiWarps * kEpiStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &tail->abort_flag;
 
@@ -229,7 +249,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(smem_u32(&tail->tmem_full[a]), 1);
-      mbar_init(smem_u32(&tail->tmem_empty[a]), 4);   // one arrival per epilogue warp
+      mbar_init(smem_u32(&tail->tmem_empty[a]), kEpiWarps);   // one arrival per epilogue warp
     }
     tail->abort_flag = 0;
     fence_barrier_init();
@@ -291,8 +311,8 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         const TileCoord c = tile_coord(tail, p.n_groups, p.n_tiles_n, tile);
-        const int brow0 = c.expert * p.b_rows_per_expert + (p.swiglu ? c.nt * p.bn : c.nt * 2 * p.bn);
-        const int brow1 = p.swiglu ? brow0 : brow0 + p.bn;
+        const int brow0 = c.expert * p.b_rows_per_expert + (SWIGLU ? c.nt * p.bn : c.nt * 2 * p.bn);
+        const int brow1 = SWIGLU ? brow0 : brow0 + p.bn;
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
           if (!(ok = mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status))) break;
           const uint32_t full = smem_u32(&tail->full[stage]);
@@ -341,9 +361,15 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
     }
   } else {
-    // ---- epilogue: TMEM -> registers -> global ----------------------------------------------
-    const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const int row_local = q * 32 + lane;
+    // ---- epilogue: TMEM -> registers -> bf16 -> (warp-private smem transpose) -> global -------
+    // A thread owns one accumulator row, so storing straight from registers would scatter 16-byte
+    // pieces over 32 rows per instruction.  Instead each warp stages 32 rows x 64 columns (128 B
+    // per row, 16-byte chunks XOR-swizzled by row) and writes them back out 4 rows per
+    // instruction: every store covers whole 128-byte lines, masked per row for ragged tiles.
+    const int q = warp & 3;                   // TMEM lane quarter this warp may read
+    const uint32_t stg = smem_u32(epi_smem + (size_t)(warp - 2) * kEpiStageBytes);
+    const int out_cols = SWIGLU ? p.bn : 2 * p.bn;
+    const int rd_row = lane >> 3, rd_chunk = lane & 7;   // read-back role: 4 rows x 8 chunks per step
     int as = 0;
     uint32_t aphase = 0;
     bool ok = true;
@@ -354,35 +380,45 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * kAccCols);
-      const bool valid = row_local < c.rows_valid;
-      const int out_cols = p.swiglu ? p.bn : 2 * p.bn;
-      __nv_bfloat16* orow = p.out + (int64_t)(c.row0 + row_local) * p.ld_out + (int64_t)c.nt * out_cols;
-      for (int col = 0; col < out_cols; col += 32) {
-        uint32_t a[32];
-        uint32_t packed[16];
-        tmem_ld32(taddr + (uint32_t)col, a);
-        if (p.swiglu) {
-          uint32_t b[32];
-          tmem_ld32(taddr + (uint32_t)(p.bn + col), b);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float h0 = silu_f(__uint_as_float(a[2 * i])) * __uint_as_float(b[2 * i]);
-            const float h1 = silu_f(__uint_as_float(a[2 * i + 1])) * __uint_as_float(b[2 * i + 1]);
-            packed[i] = pack_bf16x2(h0, h1);
+      const int rows_here = c.rows_valid - q * 32;        // valid rows among this warp's 32
+      __nv_bfloat16* obase = p.out + (int64_t)(c.row0 + q * 32) * p.ld_out + (int64_t)c.nt * out_cols;
+      uint32_t a0[32], a1[32], b0[32], b1[32], packed[32];
+      tmem_ld32(taddr, a0);
+      tmem_ld32(taddr + 32u, a1);
+      if (SWIGLU) {
+        tmem_ld32(taddr + (uint32_t)p.bn, b0);
+        tmem_ld32(taddr + (uint32_t)p.bn + 32u, b1);
+      }
+      for (int col = 0; col < out_cols; col += 64) {
+        tmem_ld_wait();
+        convert_slice<SWIGLU>(a0, b0, packed);
+        convert_slice<SWIGLU>(a1, b1, packed + 16);
+        if (col + 64 < out_cols) {           // next slice's TMEM loads fly while this one is stored
+          tmem_ld32(taddr + (uint32_t)(col + 64), a0);
+          tmem_ld32(taddr + (uint32_t)(col + 96), a1);
+          if (SWIGLU) {
+            tmem_ld32(taddr + (uint32_t)(p.bn + col + 64), b0);
+            tmem_ld32(taddr + (uint32_t)(p.bn + col + 96), b1);
           }
-        } else {
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            packed[i] = pack_bf16x2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
         }
-        if (valid) {
-          uint4* dst = reinterpret_cast<uint4*>(orow + col);
+        // row `lane`: chunk j (columns 8j..8j+7) goes to position j ^ (lane & 7)
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[i] = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(packed[4 * j]), "r"(packed[4 * j + 1]),
+                       "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
         }
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int r = it * 4 + rd_row;
+          const uint32_t addr = stg + (uint32_t)(r * 128 + ((rd_chunk ^ (r & 7)) << 4));
+          uint4 v;
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+          if (r < rows_here)
+            *reinterpret_cast<uint4*>(obase + (int64_t)r * p.ld_out + col + rd_chunk * 8) = v;
+        }
+        __syncwarp();
       }
       tc_fence_before();
       __syncwarp();
@@ -432,19 +468,24 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <bool SWIGLU>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const GemmParams& p,
+                       int grid, cudaStream_t st) {
+  static bool attr_set = false;   // per instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_grouped_gemm<SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  k_grouped_gemm<SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, p);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn) {
   if (a.n_groups == 0 || a.s_cap == 0) return FEPLB_OK;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_grouped_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) {
-      snprintf(err, errn, "cudaFuncSetAttribute(k_grouped_gemm): %s", cudaGetErrorString(e));
-      return FEPLB_E_CUDA;
-    }
-    attr_set = true;
-  }
   // pass 1: H = silu(X W1) * (X W3);  N tile = bn columns of H, MMA N = 2*bn
   const int bn1 = (a.f % 128 == 0) ? 128 : 64;
   // pass 2: Y = H W2;  N tile = 2*bn columns of Y
@@ -460,19 +501,17 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   }
   GemmParams p1;
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
-  p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1; p1.swiglu = 1;
+  p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1;
   p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status;
   GemmParams p2 = p1;
-  p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2; p2.swiglu = 0;
+  p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d;
 
-  k_grouped_gemm<<<a.num_sms, kThreads, kSmemBytes, st>>>(tm_x, tm_w1, tm_w3, p1);
+  cudaError_t e = launch_one<true>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st);
   ++*n_launch;
-  cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) {
-    k_grouped_gemm<<<a.num_sms, kThreads, kSmemBytes, st>>>(tm_h, tm_w2, tm_w2, p2);
+    e = launch_one<false>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st);
     ++*n_launch;
-    e = cudaGetLastError();
   }
   if (e != cudaSuccess) {
     snprintf(err, errn, "k_grouped_gemm launch: %s", cudaGetErrorString(e));

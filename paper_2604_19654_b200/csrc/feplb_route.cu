@@ -117,6 +117,56 @@ k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __
   if (e == 0) pad_off[E] = total;
 }
 
+// Whole-layer variant of k_scan: from the per-CTA histograms alone it produces everything the
+// rest of the pass needs -- counts, per-rank loads, segment offsets, the home group table (with
+// the dynamic-expert mask, given or derived from the counts) and the -1 tail of row_to_token --
+// so that no memset, atomic or extra launch sits between the histogram and the plan.
+__global__ void __launch_bounds__(1024)
+k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int dyn,
+             const uint8_t* __restrict__ mask_in, int32_t* __restrict__ counts_out,
+             int32_t* __restrict__ rank_load_out, int32_t* __restrict__ pad_off,
+             feplb_group* __restrict__ groups, uint8_t* __restrict__ mask_out,
+             int32_t* __restrict__ row_to_token, int64_t s_cap) {
+  __shared__ int tmp[64];
+  __shared__ int sc[FEPLB_MAX_EXPERTS];
+  const int e = threadIdx.x;
+  int c = 0;
+  if (e < E) {
+    int run = 0;
+    for (int b = 0; b < nb; ++b) {
+      const int v = block_hist[(int64_t)b * E + e];
+      block_hist[(int64_t)b * E + e] = run;
+      run += v;
+    }
+    c = run;
+    counts_out[e] = c;
+    sc[e] = c;
+  }
+  int total;
+  const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, &total);   // also orders sc[] for all threads
+  if (e < E) {
+    pad_off[e] = off;
+    int is_dyn;
+    if (mask_in) {
+      is_dyn = mask_in[e] != 0;
+    } else {
+      const int b0 = e / L * L;
+      int better = 0;
+      for (int o = b0; o < b0 + L; ++o) better += (sc[o] > c) || (sc[o] == c && o < e);
+      is_dyn = better < dyn;
+    }
+    groups[e] = feplb_group{e, off, c, e / L, is_dyn};
+    if (mask_out) mask_out[e] = (uint8_t)is_dyn;
+  }
+  if (e == 0) pad_off[E] = total;
+  if (e < E / L) {
+    int sum = 0;
+    for (int o = e * L; o < (e + 1) * L; ++o) sum += sc[o];
+    rank_load_out[e] = sum;
+  }
+  for (int64_t i = (int64_t)total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
+}
+
 // Stable rank of every slot: slot_to_row[s] and row_to_token[row].
 __global__ void __launch_bounds__(kThreads)
 k_rank(const int32_t* __restrict__ ids, int64_t S, int K, int E, const int32_t* __restrict__ block_base,
@@ -200,9 +250,11 @@ k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, u
 // Zero the padding rows at the end of every expert's segment (row_align > 1 only).
 __global__ void __launch_bounds__(kThreads)
 k_zero_pad(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_off, uint4* __restrict__ x_perm,
-           int chunks) {
+           int chunks, int32_t* __restrict__ row_to_token) {
   const int e = blockIdx.x;
   const int64_t r0 = (int64_t)pad_off[e] + counts[e], r1 = pad_off[e + 1];
+  if (row_to_token)
+    for (int64_t r = r0 + threadIdx.x; r < r1; r += kThreads) row_to_token[r] = -1;
   const int64_t n = (r1 - r0) * chunks;
   uint4* p = x_perm + r0 * chunks;
   const uint4 z = make_uint4(0, 0, 0, 0);
@@ -276,11 +328,11 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
 
 cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
                                 const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                cudaStream_t st, int64_t* n_launch) {
+                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token) {
   cudaError_t err;
   const int chunks = d / 8;
   if (A > 1) {
-    k_zero_pad<<<E, kThreads, 0, st>>>(counts, pad_off, (uint4*)x_perm, chunks);
+    k_zero_pad<<<E, kThreads, 0, st>>>(counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token);
     ++*n_launch;
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
@@ -297,6 +349,34 @@ cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
                                      feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch) {
   k_home_groups<<<1, 1024, 0, st>>>(counts, mask_in, E, E / R, A, dyn, groups, mask_out);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R, int A, int dyn,
+                                     const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
+                                     int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
+                                     int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                     cudaStream_t st, int64_t* n_launch) {
+  cudaError_t err;
+  const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
+  if (nb) {
+    k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E, block_hist, nullptr, nullptr, status);
+    ++*n_launch;
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  }
+  k_scan_fused<<<1, 1024, 0, st>>>(block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off, groups,
+                                   mask_out, row_to_token, s_cap);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
+                              const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,
+                              cudaStream_t st, int64_t* n_launch) {
+  const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
+  if (!nb) return cudaSuccess;
+  k_rank<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, K, E, block_base, pad_off, slot_to_row, row_to_token, s_cap);
   ++*n_launch;
   return cudaGetLastError();
 }
