@@ -360,7 +360,7 @@ extern "C" int feplb_combine(feplb_ctx* c, const void* y_perm, const int32_t* sl
   int rc = check_dev_ptrs(c, {y_perm, out});
   if (rc != FEPLB_OK) return rc;
   if (!slot_to_row || !gates) return fail(c, FEPLB_E_INVALID, "combine: null pointer");
-  CUDA_TRY(c, feplb_launch_combine(y_perm, slot_to_row, gates, out, c->cfg.T, c->cfg.K, c->cfg.d,
+  CUDA_TRY(c, feplb_launch_combine(y_perm, slot_to_row, gates, out, c->cfg.T, c->cfg.K, c->cfg.d, c->num_sms,
                                    (cudaStream_t)stream, &c->launches));
   return FEPLB_OK;
 }

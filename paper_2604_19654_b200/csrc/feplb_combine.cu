@@ -30,55 +30,67 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-__global__ void __launch_bounds__(kThreads)
+// Work unit = (token, 32-chunk slice of its row) = 512 output bytes; the units are dealt out in
+// equal contiguous ranges to all warps of a grid sized to the machine, so that no tail wave forms.
+__global__ void __launch_bounds__(kThreads, 3)
 k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_to_row,
           const float* __restrict__ gates, uint4* __restrict__ out, int T, int K, int chunks) {
+  // launched with programmatic stream serialization: CTAs may become resident while the expert
+  // GEMM before them drains; its y_perm is complete only after this wait
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int lane = threadIdx.x & 31;
-  const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
-  const int nwarps = (gridDim.x * kThreads) >> 5;
-  for (int t = warp; t < T; t += nwarps) {
-    int myrow = -1;
-    float myg = 0.f;
-    if (lane < K) {
-      myrow = slot_to_row[(int64_t)t * K + lane];
-      myg = gates[(int64_t)t * K + lane];
+  const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int slices = (chunks + 31) / 32;
+  const int64_t units = (int64_t)T * slices;
+  const int64_t u0 = units * warp / nwarps, u1 = units * (warp + 1) / nwarps;
+  int cur_t = -1, myrow = -1;
+  float myg = 0.f;
+  for (int64_t u = u0; u < u1; ++u) {
+    const int t = (int)(u / slices);
+    const int c = (int)(u - (int64_t)t * slices) * 32 + lane;
+    if (t != cur_t) {            // warp-uniform
+      cur_t = t;
+      myrow = -1;
+      myg = 0.f;
+      if (lane < K) {
+        myrow = slot_to_row[(int64_t)t * K + lane];
+        myg = gates[(int64_t)t * K + lane];
+      }
     }
-    for (int c0 = 0; c0 < chunks; c0 += 32) {
-      const int c = c0 + lane;
-      const bool on = c < chunks;
-      float acc[8];
+    const bool on = c < chunks;
+    float acc[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-      for (int k0 = 0; k0 < K; k0 += kBatch) {
-        uint4 v[kBatch];
-        float g[kBatch];
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += kBatch) {
+      uint4 v[kBatch];
+      float g[kBatch];
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-          const int k = k0 + j;
-          const int row = __shfl_sync(0xffffffffu, myrow, k & 31);
-          g[j] = __shfl_sync(0xffffffffu, myg, k & 31);
-          v[j] = make_uint4(0, 0, 0, 0);
-          if (k >= K || row < 0) g[j] = 0.f;
-          else if (on) v[j] = ld_nc_v4(y_perm + (int64_t)row * chunks + c);
-        }
+      for (int j = 0; j < kBatch; ++j) {
+        const int k = k0 + j;
+        const int row = __shfl_sync(0xffffffffu, myrow, k & 31);
+        g[j] = __shfl_sync(0xffffffffu, myg, k & 31);
+        v[j] = make_uint4(0, 0, 0, 0);
+        if (k >= K || row < 0) g[j] = 0.f;
+        else if (on) v[j] = ld_nc_v4(y_perm + (int64_t)row * chunks + c);
+      }
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-          if (k0 + j < K) {
-            fma_bf16x2(acc[0], acc[1], g[j], v[j].x);
-            fma_bf16x2(acc[2], acc[3], g[j], v[j].y);
-            fma_bf16x2(acc[4], acc[5], g[j], v[j].z);
-            fma_bf16x2(acc[6], acc[7], g[j], v[j].w);
-          }
+      for (int j = 0; j < kBatch; ++j) {
+        if (k0 + j < K) {
+          fma_bf16x2(acc[0], acc[1], g[j], v[j].x);
+          fma_bf16x2(acc[2], acc[3], g[j], v[j].y);
+          fma_bf16x2(acc[4], acc[5], g[j], v[j].z);
+          fma_bf16x2(acc[6], acc[7], g[j], v[j].w);
         }
       }
-      if (on) {
-        uint4 o;
-        o.x = pack_bf16x2(acc[0], acc[1]);
-        o.y = pack_bf16x2(acc[2], acc[3]);
-        o.z = pack_bf16x2(acc[4], acc[5]);
-        o.w = pack_bf16x2(acc[6], acc[7]);
-        out[(int64_t)t * chunks + c] = o;
-      }
+    }
+    if (on) {
+      uint4 o;
+      o.x = pack_bf16x2(acc[0], acc[1]);
+      o.y = pack_bf16x2(acc[2], acc[3]);
+      o.z = pack_bf16x2(acc[4], acc[5]);
+      o.w = pack_bf16x2(acc[6], acc[7]);
+      out[(int64_t)t * chunks + c] = o;
     }
   }
 }
@@ -86,13 +98,22 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_to_
 }  // namespace
 
 cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row, const float* gates, void* out,
-                                 int T, int K, int d, cudaStream_t st, int64_t* n_launch) {
+                                 int T, int K, int d, int num_sms, cudaStream_t st, int64_t* n_launch) {
   if (T == 0) return cudaSuccess;
-  const int warps_per_block = kThreads / 32;
-  int blocks = (T + warps_per_block - 1) / warps_per_block;
-  const int max_blocks = 148 * 8;
-  if (blocks > max_blocks) blocks = max_blocks;
-  k_combine<<<blocks, kThreads, 0, st>>>((const uint4*)y_perm, slot_to_row, gates, (uint4*)out, T, K, d / 8);
+  // a grid that fills every SM exactly once at 3 CTAs per SM (fewer CTAs if there is less work)
+  const int64_t units = (int64_t)T * ((d / 8 + 31) / 32);
+  int blocks = num_sms * 3;
+  const int64_t need = (units + kThreads / 32 - 1) / (kThreads / 32);
+  if (need < blocks) blocks = (int)need;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
   ++*n_launch;
-  return cudaGetLastError();
+  return cudaLaunchKernelEx(&cfg, k_combine, (const uint4*)y_perm, slot_to_row, gates, (uint4*)out, T, K, d / 8);
 }

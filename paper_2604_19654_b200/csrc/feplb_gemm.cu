@@ -238,6 +238,10 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &tail->abort_flag;
 
+  // Programmatic dependent launch: the next kernel of the stream may be scheduled as soon as SMs
+  // free up (its set-up then overlaps this grid's tail); it waits for this grid's results itself.
+  asm volatile("griddepcontrol.launch_dependents;");
+
   // ---- set-up: barriers, TMEM, group table ------------------------------------------------
   if (threadIdx.x == 0) {
     prefetch_tmap(&tm_a);
@@ -259,6 +263,9 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
     tmem_relinquish();
   }
+  // everything above touched only this CTA's resources; from here on the results of the kernels
+  // before this one (rows, group table) are read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int g = threadIdx.x; g < p.n_groups; g += kThreads) {
     const feplb_group gr = p.groups[g];
     const bool selected = p.which == FEPLB_FFN_ALL || (p.which == FEPLB_FFN_STATIC) == (gr.is_dynamic == 0);
@@ -478,8 +485,17 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUte
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  k_grouped_gemm<SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU>, ta, tb0, tb1, p);
 }
 
 }  // namespace

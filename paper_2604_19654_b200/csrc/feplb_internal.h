@@ -51,7 +51,7 @@ cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
                                      feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row, const float* gates, void* out,
-                                 int T, int K, int d, cudaStream_t st, int64_t* n_launch);
+                                 int T, int K, int d, int num_sms, cudaStream_t st, int64_t* n_launch);
 
 struct feplb_gemm_args {
   const void* x_perm; const void* w1; const void* w3; const void* w2;

@@ -217,31 +217,40 @@ __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
 // Row gather, token-major: one warp reads a token's row once (16-byte vectors, coalesced) and
 // writes it to the K rows its slots were ranked to.
 constexpr int kGatherUnroll = 4;
+// Work unit = (token, slice of 4 x 32 chunks = 2 KiB of its row); equal contiguous ranges of units
+// per warp over a grid sized to the machine, so that no tail wave forms.
 __global__ void __launch_bounds__(kThreads)
 k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, uint4* __restrict__ x_perm,
          int T, int K, int chunks) {
   const int lane = threadIdx.x & 31;
-  const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
-  const int nwarps = (gridDim.x * kThreads) >> 5;
-  for (int t = warp; t < T; t += nwarps) {
-    const int myrow = lane < K ? slot_to_row[(int64_t)t * K + lane] : -1;
+  const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int slices = (chunks + 32 * kGatherUnroll - 1) / (32 * kGatherUnroll);
+  const int64_t units = (int64_t)T * slices;
+  const int64_t u0 = units * warp / nwarps, u1 = units * (warp + 1) / nwarps;
+  int cur_t = -1, myrow = -1;
+  for (int64_t u = u0; u < u1; ++u) {
+    const int t = (int)(u / slices);
+    const int c0 = (int)(u - (int64_t)t * slices) * 32 * kGatherUnroll;
+    if (t != cur_t) {            // warp-uniform
+      cur_t = t;
+      myrow = lane < K ? slot_to_row[(int64_t)t * K + lane] : -1;
+    }
     const uint4* src = x + (int64_t)t * chunks;
-    for (int c0 = 0; c0 < chunks; c0 += 32 * kGatherUnroll) {
-      uint4 v[kGatherUnroll];
+    uint4 v[kGatherUnroll];
 #pragma unroll
-      for (int u = 0; u < kGatherUnroll; ++u) {
-        const int c = c0 + u * 32 + lane;
-        if (c < chunks) v[u] = ld_nc_v4(src + c);
-      }
-      for (int k = 0; k < K; ++k) {
-        const int row = __shfl_sync(0xffffffffu, myrow, k);
-        if (row < 0) continue;
-        uint4* dst = x_perm + (int64_t)row * chunks;
+    for (int i = 0; i < kGatherUnroll; ++i) {
+      const int c = c0 + i * 32 + lane;
+      if (c < chunks) v[i] = ld_nc_v4(src + c);
+    }
+    for (int k = 0; k < K; ++k) {
+      const int row = __shfl_sync(0xffffffffu, myrow, k);
+      if (row < 0) continue;
+      uint4* dst = x_perm + (int64_t)row * chunks;
 #pragma unroll
-        for (int u = 0; u < kGatherUnroll; ++u) {
-          const int c = c0 + u * 32 + lane;
-          if (c < chunks) dst[c] = v[u];
-        }
+      for (int i = 0; i < kGatherUnroll; ++i) {
+        const int c = c0 + i * 32 + lane;
+        if (c < chunks) dst[c] = v[i];
       }
     }
   }
@@ -337,10 +346,10 @@ cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
   if (T == 0) return cudaSuccess;
-  const int warps_per_block = kThreads / 32;
-  int blocks = (T + warps_per_block - 1) / warps_per_block;
-  const int max_blocks = 148 * 8;
-  if (blocks > max_blocks) blocks = max_blocks;
+  const int64_t units = (int64_t)T * ((chunks + 32 * kGatherUnroll - 1) / (32 * kGatherUnroll));
+  int blocks = 148 * 8;   // 8 CTAs of 256 threads per SM are resident
+  const int64_t need = (units + kWarps - 1) / kWarps;
+  if (need < blocks) blocks = (int)need;
   k_gather<<<blocks, kThreads, 0, st>>>((const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
   ++*n_launch;
   return cudaGetLastError();
