@@ -34,6 +34,8 @@ struct feplb_ctx {
   int nb = 0;   // CTAs of the permutation kernels
   char err[512] = {0};
   int64_t launches = 0;
+  int gemm_pair_default = 0;   // GEMM form for launches whose group sizes the host does not know
+  int gemm_pair_forced = -1;   // FEPLB_GEMM_PAIR=0/1 forces one form everywhere (experiments, tests)
 
   // device scratch
   int32_t* d_block_hist = nullptr;
@@ -71,6 +73,7 @@ struct feplb_ctx {
   const uint8_t* job_mask = nullptr;
   int job_rc = FEPLB_OK;
   int n_dyn_groups = 0;
+  int dyn_pair = 0;   // GEMM form chosen by the planner for the dynamic groups (it knows their sizes)
   // plan storage owned by the context
   std::vector<feplb_move> moves;
   std::vector<feplb_group> groups;
@@ -138,6 +141,9 @@ void planner_main(feplb_ctx* c) {
         for (int i = 0; i < c->plan.n_groups; ++i)
           if (c->plan.groups[i].is_dynamic) c->h_dyn_groups[n++] = c->plan.groups[i];
         c->n_dyn_groups = n;
+        int64_t dyn_rows = 0;
+        for (int i = 0; i < n; ++i) dyn_rows += c->h_dyn_groups[i].rows;
+        c->dyn_pair = c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (n > 0 && dyn_rows >= (int64_t)512 * n);
         cudaError_t e = cudaSuccess;
         if (n) e = cudaMemcpyAsync(c->d_dyn_groups, c->h_dyn_groups, sizeof(feplb_group) * n, cudaMemcpyHostToDevice, c->copy_stream);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_plan, c->copy_stream);
@@ -194,6 +200,9 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   c->device = dev;
   c->num_sms = prop.multiProcessorCount;
   c->s_cap = feplb_s_pad(cfg);
+  // 256-row pair tiles pay off when an expert's segment is several tiles long on average
+  c->gemm_pair_default = (int64_t)cfg->T * cfg->K >= (int64_t)2048 * cfg->E;
+  if (const char* e = getenv("FEPLB_GEMM_PAIR")) c->gemm_pair_default = c->gemm_pair_forced = atoi(e) != 0;
   const int64_t S = (int64_t)cfg->T * cfg->K;
   c->nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   const int cap_moves = cfg->R * cfg->max_num_dyn;
@@ -330,7 +339,9 @@ extern "C" int feplb_home_groups(feplb_ctx* c, const int32_t* counts, const uint
 }
 
 static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void* w3, const void* w2,
-                    const feplb_group* groups, int32_t n_groups, int32_t which, void* h, void* y, cudaStream_t st) {
+                    const feplb_group* groups, int32_t n_groups, int32_t which, void* h, void* y, cudaStream_t st,
+                    int pair = -1) {
+  if (pair < 0) pair = c->gemm_pair_default;
   if (n_groups < 0 || n_groups > FEPLB_MAX_GROUPS) return fail(c, FEPLB_E_INVALID, "expert_ffn: n_groups out of range");
   if (which != FEPLB_FFN_ALL && which != FEPLB_FFN_STATIC && which != FEPLB_FFN_DYNAMIC)
     return fail(c, FEPLB_E_INVALID, "expert_ffn: bad selector");
@@ -342,7 +353,7 @@ static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void
   a.x_perm = x_perm; a.w1 = w1; a.w3 = w3; a.w2 = w2; a.h = h; a.y = y;
   a.groups = groups; a.n_groups = n_groups; a.which = which;
   a.E = c->cfg.E; a.d = c->cfg.d; a.f = c->cfg.f; a.s_cap = (int64_t)c->s_cap;
-  a.status = c->d_status; a.num_sms = c->num_sms;
+  a.status = c->d_status; a.num_sms = c->num_sms; a.pair = pair;
   return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err));
 }
 
@@ -518,7 +529,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   if (rc != FEPLB_OK) return rc;
   if (rc_join != FEPLB_OK) return rc_join;
   TL_EVENT(EV_DYN0);
-  if ((rc = ffn_impl(c, x_perm, w1, w3, w2, dyn_groups, n_dyn, FEPLB_FFN_ALL, h_scratch, y_perm, st)) != FEPLB_OK) return rc;
+  if ((rc = ffn_impl(c, x_perm, w1, w3, w2, dyn_groups, n_dyn, FEPLB_FFN_ALL, h_scratch, y_perm, st, c->dyn_pair)) != FEPLB_OK) return rc;
   TL_EVENT(EV_DYN1);
   // step 6
   if ((rc = feplb_combine(c, y_perm, slot_to_row, gates, out, stream)) != FEPLB_OK) return rc;

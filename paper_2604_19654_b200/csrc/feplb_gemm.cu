@@ -33,18 +33,33 @@ constexpr int kABytes = BM * BK * 2;               // 16 KiB per sub-tile
 constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
 constexpr unsigned long long kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s per wait
 
-// Tile 128 x 256 (UMMA M x N), K step 64: 4 stages of 48 KiB (A 16 KiB + B 32 KiB); two
-// accumulators in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1.
-constexpr int kStages = 4;
+// Two forms of one kernel.
+//   single (PAIR = false): one CTA computes a 128 x 256 tile (UMMA M x N, cta_group::1); K step 64;
+//     4 stages of 48 KiB (A 16 KiB + B 32 KiB).  The mainloop needs 96 bytes per MMA cycle from L2.
+//   pair (PAIR = true): a cluster of two CTAs computes a 256 x 256 tile with cta_group::2 MMAs
+//     issued by the even CTA: each CTA stages its own 128 rows of A and HALF of the B tile (the
+//     W1 tile in the even CTA and the W3 tile in the odd one in pass 1), so a CTA needs only
+//     64 bytes per MMA cycle from L2 and the ring holds 6 stages of 32 KiB.  No multicast: each
+//     CTA loads its own halves.  Used for launches whose groups are large (a 256-row tile wastes
+//     more on a ragged tail).
+// Both keep two accumulators in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1.
+template <bool PAIR> struct Ring {
+  static constexpr int kStages = PAIR ? 6 : 4;
+  static constexpr int kStageBytes = kABytes + (PAIR ? kBBytesMax / 2 : kBBytesMax);   // multiple of 1024
+  static constexpr int kTileRows = PAIR ? 2 * BM : BM;
+};
+constexpr int kMaxStages = 6;
 constexpr int kAccStages = 2;
-constexpr int kStageBytes = kABytes + kBBytesMax;   // 48 KiB, a multiple of 1024
+constexpr int kRingBytes = 4 * (kABytes + kBBytesMax);   // 192 KiB in both forms
+static_assert(Ring<false>::kStages * Ring<false>::kStageBytes == kRingBytes &&
+              Ring<true>::kStages * Ring<true>::kStageBytes == kRingBytes, "ring size");
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kEpiStageBytes = 32 * 128;            // per epilogue warp: 32 rows x 64 bf16
 
 struct SmemTail {
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kAccStages];
   unsigned long long tmem_empty[kAccStages];
   uint32_t tmem_base;
@@ -54,7 +69,7 @@ struct SmemTail {
   int g_rows[FEPLB_MAX_GROUPS];
   int g_expert[FEPLB_MAX_GROUPS];
 };
-constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kStages * kStageBytes +
+constexpr size_t kSmemBytes = 1024 /* alignment slack */ + (size_t)kRingBytes +
                               (size_t)kEpiWarps * kEpiStageBytes + sizeof(SmemTail);
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 static_assert(kSmemBytes > 116 * 1024, "two CTAs must never share an SM: each allocates all of TMEM");
@@ -173,6 +188,54 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- cluster-of-two forms (cta_group::2) --------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose byte count is credited to an mbarrier that may
+// live in the peer CTA of the pair (cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[256 rows, 128 per CTA] * B[N columns, N/2 per CTA]
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// One arrival on the mbarrier at this offset in BOTH CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) wide and
 // 128-byte swizzled, 8-row groups 1024 bytes apart: start address >> 4 in bits [0,14), leading
 // byte offset (unused for swizzled K-major) = 1 in [16,30), stride byte offset 1024 >> 4 in
@@ -197,6 +260,7 @@ struct TileCoord { int row0, rows_valid, expert, nt; };
 
 // tile -> (group, M tile, N tile); N tiles of one M tile are consecutive so that CTAs running at
 // the same time share the A rows and sweep one expert's weights together (both stay in L2).
+template <int kRows>
 __device__ __forceinline__ TileCoord tile_coord(const SmemTail* t, int n_groups, int n_tiles_n, int tile) {
   const int mt = tile / n_tiles_n;
   int lo = 0, hi = n_groups;   // largest g with prefix[g] <= mt
@@ -206,8 +270,8 @@ __device__ __forceinline__ TileCoord tile_coord(const SmemTail* t, int n_groups,
   }
   const int local = mt - t->prefix[lo];
   TileCoord c;
-  c.row0 = t->g_row_start[lo] + local * BM;
-  c.rows_valid = min(BM, t->g_rows[lo] - local * BM);
+  c.row0 = t->g_row_start[lo] + local * kRows;
+  c.rows_valid = min(kRows, t->g_rows[lo] - local * kRows);
   c.expert = t->g_expert[lo];
   c.nt = tile - mt * n_tiles_n;
   return c;
@@ -227,13 +291,20 @@ __device__ __forceinline__ void convert_slice(const uint32_t (&a)[32], const uin
   }
 }
 
-template <bool SWIGLU>
+template <bool SWIGLU, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
+  constexpr int kStages = Ring<PAIR>::kStages, kStageBytes = Ring<PAIR>::kStageBytes;
+  constexpr int kTileRows = Ring<PAIR>::kTileRows;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* epi_smem = smem + (size_t)kStages * kStageBytes;
+  uint8_t* epi_smem = smem + (size_t)kRingBytes;
+  // pair form: rank of this CTA in its cluster of two (0 = leader, issues the MMAs), work is dealt
+  // per cluster; single form: every CTA is its own leader
+  const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   SmemTail* tail = reinterpret_cast<SmemTail*>(epi_smem + (size_t)kEpiWarps * kEpiStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &tail->abort_flag;
@@ -253,15 +324,21 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(smem_u32(&tail->tmem_full[a]), 1);
-      mbar_init(smem_u32(&tail->tmem_empty[a]), kEpiWarps);   // one arrival per epilogue warp
+      // one arrival per epilogue warp (of both CTAs in the pair form: the leader's barrier collects them)
+      mbar_init(smem_u32(&tail->tmem_empty[a]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
     tail->abort_flag = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
     __syncwarp();
-    tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_u32(&tail->tmem_base), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
+      tmem_relinquish();
+    }
   }
   // everything above touched only this CTA's resources; from here on the results of the kernels
   // before this one (rows, group table) are read
@@ -273,7 +350,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (selected && gr.rows > 0) {
       const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 &&
                       (int64_t)gr.row_start + gr.rows <= p.s_cap;
-      if (ok) tiles = (gr.rows + BM - 1) / BM;
+      if (ok) tiles = (gr.rows + kTileRows - 1) / kTileRows;
       else atomicOr(p.status, FEPLB_ST_GROUP);
     }
     tail->prefix[g + 1] = tiles;   // turned into a prefix sum below
@@ -304,11 +381,12 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (lane == 0) tail->prefix[0] = 0;
   }
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tail->tmem_base;
   const int total_tiles = tail->prefix[p.n_groups] * p.n_tiles_n;
   const uint32_t b_half_bytes = (uint32_t)p.bn * BK * 2;
-  const uint32_t stage_tx = kABytes + 2 * b_half_bytes;
+  const uint32_t stage_tx = PAIR ? 2 * (kABytes + b_half_bytes) : kABytes + 2 * b_half_bytes;
 
   if (warp == 0) {
     // ---- TMA producer ---------------------------------------------------------------------
@@ -316,8 +394,8 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const TileCoord c = tile_coord(tail, p.n_groups, p.n_tiles_n, tile);
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+        const TileCoord c = tile_coord<kTileRows>(tail, p.n_groups, p.n_tiles_n, tile);
         const int brow0 = c.expert * p.b_rows_per_expert + (SWIGLU ? c.nt * p.bn : c.nt * 2 * p.bn);
         const int brow1 = SWIGLU ? brow0 : brow0 + p.bn;
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
@@ -325,10 +403,19 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const uint32_t full = smem_u32(&tail->full[stage]);
           const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
           const uint32_t sb = sa + kABytes;
-          mbar_expect_tx(full, stage_tx);
-          tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
-          tma_load_2d(sb, &tm_b0, full, kb * BK, brow0);
-          tma_load_2d(sb + b_half_bytes, &tm_b1, full, kb * BK, brow1);
+          if (PAIR) {
+            // both CTAs credit the LEADER's barrier; the leader announces the bytes of both
+            const uint32_t full0 = map_to_cta(full, 0);
+            if (cta_rank == 0) mbar_expect_tx(full, stage_tx);
+            tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
+            if (cta_rank == 0) tma_load_2d_pair(sb, &tm_b0, full0, kb * BK, brow0);
+            else tma_load_2d_pair(sb, &tm_b1, full0, kb * BK, brow1);
+          } else {
+            mbar_expect_tx(full, stage_tx);
+            tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
+            tma_load_2d(sb, &tm_b0, full, kb * BK, brow0);
+            tma_load_2d(sb + b_half_bytes, &tm_b1, full, kb * BK, brow1);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -339,12 +426,12 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
   } else if (warp == 1) {
     // ---- MMA issuer -------------------------------------------------------------------------
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(BM, 2 * p.bn);
+    if (lane == 0 && cta_rank == 0) {
+      const uint32_t idesc = make_idesc(kTileRows, 2 * p.bn);
       int stage = 0, as = 0;
       uint32_t phase = 0, aphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
         if (!(ok = mbar_wait(smem_u32(&tail->tmem_empty[as]), aphase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * kAccCols);
@@ -357,13 +444,18 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // +32 bytes (>> 4 = 2) per K step inside the 128-byte swizzle row
-            umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+            if (PAIR) umma_bf16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+            else umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
           }
-          umma_commit(smem_u32(&tail->empty[stage]));   // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR) umma_commit_pair(smem_u32(&tail->empty[stage]));
+          else umma_commit(smem_u32(&tail->empty[stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&tail->tmem_full[as]));     // accumulator complete
+        // accumulator complete (announced to the epilogue warps of both CTAs of a pair)
+        if (PAIR) umma_commit_pair(smem_u32(&tail->tmem_full[as]));
+        else umma_commit(smem_u32(&tail->tmem_full[as]));
         if (++as == kAccStages) { as = 0; aphase ^= 1u; }
       }
     }
@@ -380,15 +472,16 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int as = 0;
     uint32_t aphase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const TileCoord c = tile_coord(tail, p.n_groups, p.n_tiles_n, tile);
+    for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+      const TileCoord c = tile_coord<kTileRows>(tail, p.n_groups, p.n_tiles_n, tile);
       ok = mbar_wait(smem_u32(&tail->tmem_full[as]), aphase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * kAccCols);
-      const int rows_here = c.rows_valid - q * 32;        // valid rows among this warp's 32
-      __nv_bfloat16* obase = p.out + (int64_t)(c.row0 + q * 32) * p.ld_out + (int64_t)c.nt * out_cols;
+      const int row_off = (int)cta_rank * BM + q * 32;    // this warp's first row inside the tile
+      const int rows_here = c.rows_valid - row_off;       // valid rows among this warp's 32
+      __nv_bfloat16* obase = p.out + (int64_t)(c.row0 + row_off) * p.ld_out + (int64_t)c.nt * out_cols;
       uint32_t a0[32], a1[32], b0[32], b1[32], packed[32];
       tmem_ld32(taddr, a0);
       tmem_ld32(taddr + 32u, a1);
@@ -429,7 +522,10 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tail->tmem_empty[as]), 0));
+        else mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      }
       if (++as == kAccStages) { as = 0; aphase ^= 1u; }
     }
   }
@@ -437,10 +533,12 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // ---- teardown ---------------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory: leave together
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -475,27 +573,44 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool SWIGLU>
+template <bool SWIGLU, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const GemmParams& p,
-                       int grid, cudaStream_t st) {
-  static bool attr_set = false;   // per instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_grouped_gemm<SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+                       int num_sms, cudaStream_t st) {
+  static int grid = 0;   // per instantiation: set on first use
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU>, ta, tb0, tb1, p);
+  if (PAIR) {
+    at[1].id = cudaLaunchAttributeClusterDimension;
+    at[1].val.clusterDim.x = 2;
+    at[1].val.clusterDim.y = 1;
+    at[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
+  if (!grid) {
+    cudaError_t e = cudaFuncSetAttribute(k_grouped_gemm<SWIGLU, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    int g = num_sms;
+    if (PAIR) {
+      // as many clusters of two as can be resident at once (one CTA per SM, both SMs in one GPC)
+      int n_clusters = 0;
+      cfg.gridDim = dim3(num_sms / 2 * 2);
+      e = cudaOccupancyMaxActiveClusters(&n_clusters, k_grouped_gemm<SWIGLU, PAIR>, &cfg);
+      if (e != cudaSuccess) return e;
+      if (n_clusters < 1) return cudaErrorLaunchOutOfResources;
+      g = 2 * (n_clusters < num_sms / 2 ? n_clusters : num_sms / 2);
+    }
+    grid = g;
+  }
+  cfg.gridDim = dim3(grid);
+  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, p);
 }
 
 }  // namespace
@@ -523,10 +638,12 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d;
 
-  cudaError_t e = launch_one<true>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st);
+  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st)
+                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st);
   ++*n_launch;
   if (e == cudaSuccess) {
-    e = launch_one<false>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st);
+    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st)
+               : launch_one<false, false>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st);
     ++*n_launch;
   }
   if (e != cudaSuccess) {

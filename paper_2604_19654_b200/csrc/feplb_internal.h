@@ -60,6 +60,7 @@ struct feplb_gemm_args {
   int E, d, f; int64_t s_cap;
   uint32_t* status;
   int num_sms;
+  int pair;   // 1: clusters of two CTAs on 256-row tiles (cta_group::2); 0: one CTA per 128-row tile
 };
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);

@@ -132,11 +132,18 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
   const int e = threadIdx.x;
   int c = 0;
   if (e < E) {
+    // exclusive scan over CTAs, eight independent loads in flight per round (the in-place stores
+    // would otherwise serialise every load behind the previous store)
     int run = 0;
-    for (int b = 0; b < nb; ++b) {
-      const int v = block_hist[(int64_t)b * E + e];
-      block_hist[(int64_t)b * E + e] = run;
-      run += v;
+    for (int b0 = 0; b0 < nb; b0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = b0 + j < nb ? block_hist[(int64_t)(b0 + j) * E + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (b0 + j < nb) block_hist[(int64_t)(b0 + j) * E + e] = run;
+        run += v[j];
+      }
     }
     c = run;
     counts_out[e] = c;
