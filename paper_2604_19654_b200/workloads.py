@@ -81,6 +81,10 @@ WORKLOADS = {
     "cfg3-smooth": Workload("cfg3-smooth", 3, T=16384, d=6144, f=2048, E=128, K=8, R=8, dyn=4,
                             max_num_dyn=8, tau=64, n_microbatches=16, routing="dirichlet",
                             alpha=0.2, smooth=0.5),
+    # The GLM-5-like expert shapes on a device footprint small enough for a full ncu capture
+    # (2.25 GiB of weights, ~1 GiB of activations); 1024 rows per expert on average like cfg3.
+    "cfg3-prof": Workload("cfg3-prof", 3, T=4096, d=6144, f=2048, E=32, K=8, R=4, dyn=4, max_num_dyn=8,
+                          tau=64, n_microbatches=2, routing="dirichlet", alpha=0.2),
     # Extreme skew: 3 experts of one rank take 35 % of all (token, k) slots.
     "cfg4": Workload("cfg4", 4, T=4096, d=2048, f=768, E=64, K=6, R=4, dyn=4, max_num_dyn=8,
                      tau=64, n_microbatches=8, routing="hot3", alpha=0.35),
