@@ -31,7 +31,7 @@ METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 # DRAM bytes (read + write) of one k_grouped_gemm launch at the benchmarked workload, from the ncu
 # capture summarised under profiles/; None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 190.0e6}   # profiles/k_grouped_gemm_cfg2.md: 760 MB over the 4 launches
 
 
 def _peaks():
@@ -280,27 +280,33 @@ def _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world,
     for x, i, g in host:
         pinned.append((torch.from_numpy(x.view(np.int16)).pin_memory(), torch.from_numpy(i).pin_memory(),
                        torch.from_numpy(g).pin_memory()))
-    out_host = torch.empty(w.T, w.d, dtype=torch.int16).pin_memory()
-    x_dev = torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda")
-    i_dev = torch.empty(w.T, w.K, dtype=torch.int32, device="cuda")
-    g_dev = torch.empty(w.T, w.K, dtype=torch.float32, device="cuda")
+    # two staging slots: the copies of micro-batch i+1 overlap the kernels of micro-batch i
+    out_host = [torch.empty(w.T, w.d, dtype=torch.int16).pin_memory() for _ in range(2)]
+    x_dev = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    i_dev = [torch.empty(w.T, w.K, dtype=torch.int32, device="cuda") for _ in range(2)]
+    g_dev = [torch.empty(w.T, w.K, dtype=torch.float32, device="cuda") for _ in range(2)]
+    o_dev = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
 
     def step_host(i):
+        s = i & 1
         xh, ih, gh = pinned[i % n_mb]
-        ctx.moe_forward_host(xh, ih, gh, x_dev, i_dev, g_dev, d_w1, d_w3, d_w2, buf, out_host, stream=stream)
+        ctx.host_wait(s)                     # the slot's previous result has reached its host buffer
+        ctx.moe_forward_host_async(s, xh, ih, gh, x_dev[s], i_dev[s], g_dev[s], d_w1, d_w3, d_w2, buf,
+                                   o_dev[s], out_host[s], stream=stream)
 
-    for i in range(3):
+    for i in range(4):
         step_host(i)
+    ctx.host_wait(0)
+    ctx.host_wait(1)
     barrier()
     t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
     for i in range(args.steps):
         step_host(i)
-    e1.record(stream)
+    ctx.host_wait(0)
+    ctx.host_wait(1)                         # every result is in host memory
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
     barrier()
-    e2e_ms = max(e0.elapsed_time(e1), 0.0)
-    del t0
     return whole_job_throughput(world, args.steps, w.T, max_over_ranks(e2e_ms, world, "cuda"))
 
 

@@ -251,6 +251,23 @@ int feplb_moe_forward_host(feplb_ctx* ctx, const void* x_host, const int32_t* to
                            int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
                            feplb_plan_out* plan_copy, void* stream);
 
+/* Pipelined form of feplb_moe_forward_host for back-to-back micro-batches.  `slot` (0 or 1) names
+ * one of two caller-owned staging sets (x_dev, ids_dev, gates_dev, out_dev and the host buffers
+ * must differ between the two slots; the other buffers are shared).  The call copies the inputs
+ * on the context's input stream, runs the forward on `stream` once they have arrived, copies the
+ * result to out_host on the context's output stream, and returns without waiting for any of it
+ * (it still blocks briefly for the planner, like feplb_moe_forward).  So the copies of micro-batch
+ * i+1 overlap the kernels of micro-batch i.  Before reusing a slot's host buffers, or reading
+ * out_host, call feplb_host_wait(ctx, slot). */
+int feplb_moe_forward_host_async(feplb_ctx* ctx, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
+                                 const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
+                                 const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                                 int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
+                                 int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
+                                 feplb_plan_out* plan_copy, void* stream);
+/* Blocks until the result of the last feplb_moe_forward_host_async on `slot` is in its out_host. */
+int feplb_host_wait(feplb_ctx* ctx, int32_t slot);
+
 /* Turns CUDA-event timing of the stages of feplb_moe_forward on (1) or off (0, default). */
 int feplb_set_timeline(feplb_ctx* ctx, int32_t enable);
 /* Waits for the last forward's stage events and fills *out (device fields are 0 when timing was

@@ -51,6 +51,10 @@ struct feplb_ctx {
   uint8_t* h_mask = nullptr;
 
   cudaStream_t copy_stream = nullptr;
+  // pipelined host-buffer path: input and output copy streams and per-slot events
+  cudaStream_t in_stream = nullptr, out_stream = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
   cudaEvent_t ev_counts = nullptr, ev_plan = nullptr;
   cudaEvent_t evr[kEvRing][EV_N] = {{nullptr}};
   cudaEvent_t* ev = evr[0];        // event set of the current forward
@@ -220,6 +224,12 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   ok = ok && cudaMallocHost(&c->h_mask, cfg->E) == cudaSuccess;
   ok = ok && cudaMemset(c->d_status, 0, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; ok && i < 2; ++i)
+    ok = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreate(&c->ev_counts) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
   for (int r = 0; ok && r < kEvRing; ++r)
@@ -267,6 +277,13 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFreeHost(c->h_status);
   cudaFreeHost(c->h_mask);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->in_stream) cudaStreamDestroy(c->in_stream);
+  if (c->out_stream) cudaStreamDestroy(c->out_stream);
+  for (int i = 0; i < 2; ++i) {
+    if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+    if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
+    if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+  }
   if (c->ev_counts) cudaEventDestroy(c->ev_counts);
   if (c->ev_plan) cudaEventDestroy(c->ev_plan);
   for (int r = 0; r < kEvRing; ++r)
@@ -564,6 +581,49 @@ extern "C" int feplb_moe_forward_host(feplb_ctx* c, const void* x_host, const in
   if (rc != FEPLB_OK) return rc;
   if (g.T > 0) CUDA_TRY(c, cudaMemcpyAsync(out_host, out_dev, nx, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(c, cudaStreamSynchronize(st));
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_moe_forward_host_async(feplb_ctx* c, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
+                                            const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
+                                            const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
+                                            int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch,
+                                            void* y_perm, int32_t* slot_to_row, int32_t* row_to_token, void* out_dev,
+                                            void* out_host, feplb_plan_out* plan_copy, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: slot must be 0 or 1");
+  cudaStream_t st = (cudaStream_t)stream;
+  const feplb_config& g = c->cfg;
+  const size_t nx = (size_t)g.T * g.d * 2, nk = (size_t)g.T * g.K * 4;
+  if (g.T > 0 && (!x_host || !topk_ids_host || !gates_host || !out_host || !x_dev || !ids_dev || !gates_dev || !out_dev))
+    return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: null pointer");
+  // inputs: the slot's device staging was last read by the forward that used this slot before
+  if (c->slot_used[slot]) CUDA_TRY(c, cudaStreamWaitEvent(c->in_stream, c->ev_done[slot], 0));
+  if (g.T > 0) {
+    CUDA_TRY(c, cudaMemcpyAsync(ids_dev, topk_ids_host, nk, cudaMemcpyHostToDevice, c->in_stream));
+    CUDA_TRY(c, cudaMemcpyAsync(gates_dev, gates_host, nk, cudaMemcpyHostToDevice, c->in_stream));
+    CUDA_TRY(c, cudaMemcpyAsync(x_dev, x_host, nx, cudaMemcpyHostToDevice, c->in_stream));
+  }
+  CUDA_TRY(c, cudaEventRecord(c->ev_in[slot], c->in_stream));
+  // compute: after its inputs have arrived and the slot's previous result has left out_dev
+  CUDA_TRY(c, cudaStreamWaitEvent(st, c->ev_in[slot], 0));
+  if (c->slot_used[slot]) CUDA_TRY(c, cudaStreamWaitEvent(st, c->ev_out[slot], 0));
+  int rc = feplb_moe_forward(c, x_dev, ids_dev, gates_dev, w1, w3, w2, dyn_mask_host, counts, rank_load, x_perm,
+                             h_scratch, y_perm, slot_to_row, row_to_token, out_dev, plan_copy, stream);
+  if (rc != FEPLB_OK) return rc;
+  CUDA_TRY(c, cudaEventRecord(c->ev_done[slot], st));
+  // output
+  CUDA_TRY(c, cudaStreamWaitEvent(c->out_stream, c->ev_done[slot], 0));
+  if (g.T > 0) CUDA_TRY(c, cudaMemcpyAsync(out_host, out_dev, nx, cudaMemcpyDeviceToHost, c->out_stream));
+  CUDA_TRY(c, cudaEventRecord(c->ev_out[slot], c->out_stream));
+  c->slot_used[slot] = true;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_host_wait(feplb_ctx* c, int32_t slot) {
+  if (!c) return FEPLB_E_INVALID;
+  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "host_wait: slot must be 0 or 1");
+  if (c->slot_used[slot]) CUDA_TRY(c, cudaEventSynchronize(c->ev_out[slot]));
   return FEPLB_OK;
 }
 

@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
             "feplb_plan_wait": (C.c_int, [vp, i32, C.POINTER(PlanOut), C.POINTER(vp), C.POINTER(i32), vp]),
             "feplb_moe_forward": (C.c_int, [vp] * 16 + [C.POINTER(PlanOut), vp]),
             "feplb_moe_forward_host": (C.c_int, [vp] * 20 + [C.POINTER(PlanOut), vp]),
+            "feplb_moe_forward_host_async": (C.c_int, [vp, i32] + [vp] * 19 + [C.POINTER(PlanOut), vp]),
+            "feplb_host_wait": (C.c_int, [vp, i32]),
             "feplb_set_timeline": (C.c_int, [vp, i32]),
             "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
             "feplb_timeline_totals": (C.c_int, [vp, C.POINTER(Timeline), C.POINTER(i64), i32]),
@@ -294,6 +296,20 @@ class Context:
             _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(buf.out), _ptr(out_host),
             C.byref(p.c) if p is not None else None, self._stream(stream)), "feplb_moe_forward_host")
         return p
+
+    def moe_forward_host_async(self, slot, x_host, ids_host, gates_host, x_dev, ids_dev, gates_dev, w1, w3, w2, buf,
+                               out_dev, out_host, dyn_mask_host=None, stream=None):
+        """Pipelined host-buffer forward on staging slot 0 or 1; ``host_wait(slot)`` before reading out_host."""
+        mask = None if dyn_mask_host is None else np.ascontiguousarray(dyn_mask_host, np.uint8)
+        self._chk(lib().feplb_moe_forward_host_async(
+            self._h, int(slot), _ptr(x_host), _ptr(ids_host), _ptr(gates_host), _ptr(x_dev), _ptr(ids_dev),
+            _ptr(gates_dev), _ptr(w1), _ptr(w3), _ptr(w2), _ptr(mask),
+            _ptr(buf.counts), _ptr(buf.rank_load), _ptr(buf.x_perm), _ptr(buf.h_scratch), _ptr(buf.y_perm),
+            _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(out_dev), _ptr(out_host), None,
+            self._stream(stream)), "feplb_moe_forward_host_async")
+
+    def host_wait(self, slot):
+        self._chk(lib().feplb_host_wait(self._h, int(slot)), "feplb_host_wait")
 
     def set_timeline(self, on: bool):
         self._chk(lib().feplb_set_timeline(self._h, int(bool(on))), "feplb_set_timeline")

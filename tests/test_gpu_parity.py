@@ -381,3 +381,37 @@ def test_empty_batch():
     ctx.check_status()
     assert p.moves == [] and p.groups == [] and int(buf.counts.sum()) == 0
     ctx.close()
+
+
+def test_pipelined_host_forward_matches_the_synchronous_one():
+    """Back-to-back micro-batches through the two-slot pipelined entry point give, bit for bit, what
+    the synchronous host-buffer entry point gives for each of them."""
+    torch = _torch()
+    w = W.get_workload("cfg2").with_(T=1024)
+    case = DeviceCase(w, mb=0)
+    mbs = [W.gen_microbatch(w, mb) for mb in range(5)]
+    pin = [(torch.from_numpy(x.view(np.int16)).pin_memory(), torch.from_numpy(i).pin_memory(),
+            torch.from_numpy(g).pin_memory()) for x, i, g in mbs]
+    x_dev = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    i_dev = [torch.empty(w.T, w.K, dtype=torch.int32, device="cuda") for _ in range(2)]
+    g_dev = [torch.empty(w.T, w.K, dtype=torch.float32, device="cuda") for _ in range(2)]
+    o_dev = [torch.empty(w.T, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    ref = []
+    for xh, ih, gh in pin:
+        oh = torch.zeros(w.T, w.d, dtype=torch.int16).pin_memory()
+        case.ctx.moe_forward_host(xh, ih, gh, x_dev[0], i_dev[0], g_dev[0], case.d_w1, case.d_w3, case.d_w2, case.buf, oh)
+        ref.append(oh.numpy().copy())
+    outs = [torch.zeros(w.T, w.d, dtype=torch.int16).pin_memory() for _ in pin]   # one host buffer per micro-batch
+    for n, (xh, ih, gh) in enumerate(pin):
+        s = n & 1
+        case.ctx.host_wait(s)
+        case.ctx.moe_forward_host_async(s, xh, ih, gh, x_dev[s], i_dev[s], g_dev[s], case.d_w1, case.d_w3, case.d_w2,
+                                        case.buf, o_dev[s], outs[n])
+    case.ctx.host_wait(0)
+    case.ctx.host_wait(1)
+    case.ctx.check_status()
+    for n in range(len(pin)):
+        assert np.array_equal(outs[n].numpy(), ref[n]), n
+    with pytest.raises(F.FeplbError):
+        case.ctx.host_wait(2)
+    case.close()
