@@ -273,6 +273,61 @@ def run_cuda(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """The scaling sweep (not the default bench line): cfg3's layer at T x R points, one JSON line
+    per point with tokens/s, GEMM TFLOP/s and fraction of peak, and the straggler ratios before and
+    after rebalancing.  Weights are generated once; two micro-batches per point."""
+    import torch
+    from paper_2604_19654_b200 import build as B
+    from paper_2604_19654_b200 import feplb as F
+    torch.cuda.set_device(0)
+    B.build()
+    points = W.sweep_points()
+    if args.sweep != "all":
+        keep = set(args.sweep.split(","))
+        points = [p for p in points if p.name in keep]
+    weights = W.gen_weights(points[0])
+    d_w1, d_w3, d_w2 = (F.bf16_tensor(a) for a in weights)
+    peaks = _peaks()
+    stream = torch.cuda.current_stream()
+    for w in points:
+        cfg = F.config_from_workload(w)
+        ctx, buf = F.Context(cfg), F.Buffers(cfg)
+        n_mb = 2
+        host = [W.gen_microbatch(w, mb) for mb in range(n_mb)]
+        dev = [(F.bf16_tensor(x), torch.from_numpy(i).cuda(), torch.from_numpy(g).cuda()) for x, i, g in host]
+        for i in range(3):
+            ctx.moe_forward(*dev[i % n_mb], d_w1, d_w3, d_w2, buf, want_plan=False, stream=stream)
+        ctx.check_status()
+        ctx.set_timeline(True)
+        ctx.timeline_totals(reset=True)
+        steps = max(4, min(40, int(2.0e5 / w.T)))
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for i in range(steps):
+            ctx.moe_forward(*dev[i % n_mb], d_w1, d_w3, d_w2, buf, want_plan=False, stream=stream)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1) / steps
+        totals, n_fw = ctx.timeline_totals(reset=True)
+        ctx.set_timeline(False)
+        ffn_us = (totals["dev_static_ffn_us"] + totals["dev_dynamic_ffn_us"]) / n_fw
+        tflops = gemm_flops(w) / (ffn_us * 1e-6) / 1e12
+        strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb, reps=2) if w.R > 1 else None
+        io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
+        print(json.dumps({
+            "sweep_point": w.name, "T": w.T, "R": w.R, "tokens_per_s": w.T / (ms * 1e-3), "ms_per_step": ms,
+            "gemm_tflops": tflops, "gemm_frac_of_sustained_peak": tflops / peaks["bf16_tflops_sustained"],
+            "gemm_frac_of_burst_peak": tflops / peaks["bf16_tflops"],
+            "dispatch_gbs": io_bytes / (totals["dev_dispatch_us"] / n_fw * 1e-6) / 1e9,
+            "combine_gbs": io_bytes / (totals["dev_combine_us"] / n_fw * 1e-6) / 1e9,
+            "straggler": strag}), flush=True)
+        ctx.close()
+        del buf, dev
+        torch.cuda.empty_cache()
+
+
 def _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world, n_mb):
     import torch
     import torch.distributed as dist
@@ -399,7 +454,12 @@ def main():
     ap.add_argument("--no-straggler", action="store_true")
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
+    ap.add_argument("--sweep", default=None,
+                    help='"all" or comma-separated sweep-point names (cfg5-T8192-R8, ...): prints one line per point')
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     w = W.get_workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
