@@ -92,7 +92,13 @@ WORKLOADS = {
 
 
 def get_workload(name: str) -> Workload:
-    return WORKLOADS[name]
+    """A named workload, or a point of the scaling sweep by its name (``cfg5-T8192-R8``)."""
+    if name in WORKLOADS:
+        return WORKLOADS[name]
+    for p in sweep_points():
+        if p.name == name:
+            return p
+    raise KeyError(name)
 
 
 def sweep_points(Ts=(2048, 8192, 32768, 65536), Rs=(1, 2, 4, 8, 16)):
