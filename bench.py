@@ -328,6 +328,45 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def plan_sensitivity(w, dyn, policy=1, mask="reactive", split=0, n_mb=8):
+    """Mean reduction of the token straggler (max - mean rows per rank, the paper's Section 3.1
+    metric) and mean max/mean after the plan, over ``n_mb`` micro-batches.  Host code only."""
+    from paper_2604_19654_b200 import feplb as F
+    red, after = [], []
+    for mb in range(n_mb):
+        ids, _ = W.gen_routing(w, mb)
+        counts = np.bincount(ids.ravel(), minlength=w.E).astype(np.int32)
+        if mask == "reactive":                       # the dyn busiest experts of every rank
+            m = F.select_dynamic(counts, w.E, w.R, dyn)
+        else:                                        # a fixed set: the first dyn experts of every rank
+            m = np.zeros(w.E, np.uint8)
+            for r in range(w.R):
+                m[r * w.L: r * w.L + dyn] = 1
+        p = F.plan(F.config_from_workload(w, dyn=dyn, policy=policy, split=split), counts, m)
+        b, a = p.load_before.astype(float), p.load_after.astype(float)
+        sb, sa = b.max() - b.mean(), a.max() - a.mean()
+        red.append(1.0 - sa / sb if sb > 0 else 0.0)
+        after.append(a.max() / a.mean())
+    return 100.0 * float(np.mean(red)), float(np.mean(after))
+
+
+def run_sensitivity(args):
+    """The paper's dyn sweep (Section 3.5, dyn = 2, 4, 8) plus policy / mask / split variants on
+    cfg3's routing at EP degrees 2..16; prints a markdown table.  No GPU needed."""
+    from paper_2604_19654_b200 import build as B
+    B.build()
+    base = W.get_workload("cfg3")
+    print("| R | experts/rank | dyn=2 | dyn=4 | dyn=8 | dyn=4, LITERAL | dyn=4, fixed mask | dyn=4, split |")
+    print("|---|---|---|---|---|---|---|---|")
+    for R in (2, 4, 8, 16):
+        w = base.with_(R=R)
+        cells = ["-%.0f %% (%.2f)" % plan_sensitivity(w, min(dyn, w.L)) for dyn in (2, 4, 8)]
+        cells.append("-%.0f %% (%.2f)" % plan_sensitivity(w, 4, policy=0))
+        cells.append("-%.0f %% (%.2f)" % plan_sensitivity(w, 4, mask="fixed"))
+        cells.append("-%.0f %% (%.2f)" % plan_sensitivity(w, 4, split=1))
+        print(f"| {R} | {w.L} | " + " | ".join(cells) + " |")
+
+
 def _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world, n_mb):
     import torch
     import torch.distributed as dist
@@ -456,7 +495,12 @@ def main():
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,
                     help='"all" or comma-separated sweep-point names (cfg5-T8192-R8, ...): prints one line per point')
+    ap.add_argument("--sensitivity", action="store_true",
+                    help="host-only table: straggler reduction vs dyn, policy, mask, split (no GPU)")
     args = ap.parse_args()
+    if args.sensitivity:
+        run_sensitivity(args)
+        return
     if args.sweep:
         run_sweep(args)
         return

@@ -80,3 +80,18 @@ def test_reference_arm_prints_on_rank_zero_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["config"]["workload"] == "cfg1"
+
+
+def test_dyn_sensitivity_is_monotone_and_reactive_mask_beats_fixed():
+    """The dyn sweep of the paper's Section 3.5 on synthetic routing: more dynamic experts never
+    hurt on average, and choosing the busiest experts beats a fixed set (host plan only)."""
+    import bench
+    from paper_2604_19654_b200 import workloads as W
+    w = W.get_workload("cfg3")
+    r2, _ = bench.plan_sensitivity(w, 2, n_mb=4)
+    r4, a4 = bench.plan_sensitivity(w, 4, n_mb=4)
+    r8, _ = bench.plan_sensitivity(w, 8, n_mb=4)
+    assert 0 < r2 <= r4 <= r8 <= 100
+    fixed, _ = bench.plan_sensitivity(w, 4, mask="fixed", n_mb=4)
+    literal, _ = bench.plan_sensitivity(w, 4, policy=0, n_mb=4)
+    assert fixed < r4 and literal <= r4 and a4 < 1.2
