@@ -211,7 +211,7 @@ def run_cuda(args, w):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.build()
-    cfg = F.config_from_workload(w)
+    cfg = F.config_from_workload(w, phase2_copy=1 if args.phase2 else 0)
     ctx = F.Context(cfg)
     buf = F.Buffers(cfg)
 
@@ -437,6 +437,13 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
             "cpu_baseline": cpu, "stage_us": stage_us, "straggler": strag,
         }
+        if args.phase2:   # Phase-2 weight copies on the copy engines, overlapped with the static GEMM
+            line["phase2"] = {
+                "copy_bytes_per_step": stage_us["phase2_copy_bytes"],
+                "copies_done_us_after_counts": stage_us["dev_counts_to_copies_done_us"],
+                "static_gemm_end_us_after_counts": stage_us["dev_counts_to_static_end_us"],
+                "copy_gbs": (stage_us["phase2_copy_bytes"] / max(stage_us["dev_counts_to_copies_done_us"], 1e-9) / 1e3
+                             if stage_us["phase2_copy_bytes"] else None)}
         print(json.dumps(line), flush=True)
 
 
@@ -491,6 +498,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-sample-tokens", type=int, default=1024)
     ap.add_argument("--no-straggler", action="store_true")
+    ap.add_argument("--phase2", action="store_true",
+                    help="really copy migrated experts' weights into the receive buffer (copy engines) during the static GEMM")
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,

@@ -70,13 +70,20 @@ typedef struct {
   int32_t split_granule;    /* rows; pieces of a cut expert are multiples of it */
   int32_t row_align;        /* A: expert segments of the permuted buffers start at multiples of A */
   int32_t mask_policy;      /* FEPLB_MASK_*: who chooses the dynamic experts in feplb_moe_forward */
+  int32_t phase2_copy;      /* 1: feplb_moe_forward really copies the weights of every migrated expert
+                               into a receive buffer of R*max_num_dyn slots (Section 2.2, Phase 2;
+                               Section 2.3, memory paragraph) with copy-engine transfers that overlap
+                               the static-expert GEMM, and the dynamic GEMM reads them from there.
+                               0 (default): a migration only relabels the executing rank. */
 } feplb_config;
 
 /* One copy of the plan: `rows` rows of `expert` leave home rank `src` for rank `dst`. */
 typedef struct { int32_t expert, src, dst, rows; } feplb_move;
 
 /* One segment of the grouped GEMM: rows [row_start, row_start + rows) of the permuted buffers
- * belong to `expert` and are executed on virtual rank `exec_rank`. */
+ * belong to `expert` and are executed on virtual rank `exec_rank`.  is_dynamic: 0 = static expert,
+ * 1 = dynamic expert computed with its home weights, 2 + s = dynamic expert whose weights are read
+ * from slot s of the context's receive buffer (phase2_copy). */
 typedef struct { int32_t expert, row_start, rows, exec_rank, is_dynamic; } feplb_group;
 
 /* Caller-sized plan.  cap_moves >= R*max_num_dyn and cap_groups >= E + R*max_num_dyn always
@@ -104,6 +111,8 @@ typedef struct {
   double dev_counts_to_static_start_us; /* device: counts copied -> static GEMM starts */
   double dev_counts_to_static_end_us;   /* device: counts copied -> static GEMM ends */
   double dev_total_us;
+  double dev_counts_to_copies_done_us;  /* device: counts copied -> Phase-2 weight copies landed (0 if none) */
+  double phase2_copy_bytes;             /* bytes moved by those copies */
 } feplb_timeline;
 
 typedef struct feplb_ctx feplb_ctx;

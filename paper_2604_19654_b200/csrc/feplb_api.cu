@@ -23,7 +23,7 @@ inline double us_since(clk::time_point t0) {
   return std::chrono::duration<double, std::micro>(clk::now() - t0).count();
 }
 enum JobState { JOB_IDLE = 0, JOB_PENDING = 1, JOB_RUNNING = 2, JOB_DONE = 3 };
-enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_N };
+enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_COPIES, EV_N };
 constexpr int kEvRing = 16;   // forwards whose stage events may be outstanding
 }  // namespace
 
@@ -44,6 +44,11 @@ struct feplb_ctx {
   feplb_group* d_home_groups = nullptr;
   feplb_group* d_dyn_groups = nullptr;
   uint8_t* d_mask = nullptr;
+  // Phase-2 receive buffer: R*max_num_dyn slots of one expert's weights each (phase2_copy)
+  void* d_recv_w1 = nullptr;
+  void* d_recv_w3 = nullptr;
+  void* d_recv_w2 = nullptr;
+  int n_recv_slots = 0;
   // pinned staging
   int32_t* h_counts = nullptr;
   feplb_group* h_dyn_groups = nullptr;
@@ -75,6 +80,10 @@ struct feplb_ctx {
   bool quit = false;
   int job = JOB_IDLE;
   const uint8_t* job_mask = nullptr;
+  const void* job_w1 = nullptr;   // weights of the current forward (sources of the Phase-2 copies)
+  const void* job_w3 = nullptr;
+  const void* job_w2 = nullptr;
+  double copy_bytes = 0;
   int job_rc = FEPLB_OK;
   int n_dyn_groups = 0;
   int dyn_pair = 0;   // GEMM form chosen by the planner for the dynamic groups (it knows their sizes)
@@ -145,6 +154,38 @@ void planner_main(feplb_ctx* c) {
         for (int i = 0; i < c->plan.n_groups; ++i)
           if (c->plan.groups[i].is_dynamic) c->h_dyn_groups[n++] = c->plan.groups[i];
         c->n_dyn_groups = n;
+        cudaError_t ce = cudaSuccess;
+        c->copy_bytes = 0;
+        if (cfg.phase2_copy && c->job_w1) {
+          // Phase 2 (Section 2.2): the weights of every migrated expert travel to the receiving
+          // rank's buffer on the copy engines while the SMs compute the static experts.  Move i
+          // takes the next free slot of its destination rank; the piece's group then reads slot s.
+          const int L = cfg.E / cfg.R;
+          const size_t per = (size_t)cfg.d * cfg.f * 2;
+          std::vector<int> next_slot(cfg.R, 0), move_slot(c->plan.n_moves, 0);
+          for (int i = 0; i < c->plan.n_moves && ce == cudaSuccess; ++i) {
+            const feplb_move& m = c->plan.moves[i];
+            const int s = m.dst * cfg.max_num_dyn + next_slot[m.dst]++;
+            move_slot[i] = s;
+            const char* src[3] = {(const char*)c->job_w1, (const char*)c->job_w3, (const char*)c->job_w2};
+            char* dst[3] = {(char*)c->d_recv_w1, (char*)c->d_recv_w3, (char*)c->d_recv_w2};
+            for (int k = 0; k < 3 && ce == cudaSuccess; ++k)
+              ce = cudaMemcpyAsync(dst[k] + per * s, src[k] + per * m.expert, per, cudaMemcpyDeviceToDevice, c->copy_stream);
+            c->copy_bytes += 3.0 * per;
+          }
+          std::vector<int> next_move(cfg.E, 0);   // per expert: moves consumed so far, in move order
+          for (int g = 0; g < n; ++g) {
+            feplb_group& gr = c->h_dyn_groups[g];
+            if (gr.exec_rank == gr.expert / L) continue;      // home remainder: home weights
+            int i = next_move[gr.expert];
+            while (i < c->plan.n_moves && c->plan.moves[i].expert != gr.expert) ++i;
+            next_move[gr.expert] = i + 1;
+            if (i < c->plan.n_moves) gr.is_dynamic = 2 + move_slot[i];
+          }
+          if (ce == cudaSuccess && c->copy_bytes > 0) ce = cudaEventRecord(c->ev[EV_COPIES], c->copy_stream);
+          c->tl.phase2_copy_bytes = c->copy_bytes;
+        }
+        if (ce != cudaSuccess) rc = FEPLB_E_CUDA;
         int64_t dyn_rows = 0;
         for (int i = 0; i < n; ++i) dyn_rows += c->h_dyn_groups[i].rows;
         c->dyn_pair = c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (n > 0 && dyn_rows >= (int64_t)512 * n);
@@ -218,6 +259,14 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   ok = ok && cudaMalloc(&c->d_home_groups, sizeof(feplb_group) * cfg->E) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_mask, cfg->E) == cudaSuccess;
+  if (cfg->phase2_copy && (int64_t)cfg->R * cfg->max_num_dyn > 30000) ok = false;   // slot ids travel in 15 bits
+  if (ok && cfg->phase2_copy) {
+    c->n_recv_slots = cfg->R * cfg->max_num_dyn;
+    const size_t per = (size_t)cfg->d * cfg->f * 2, n = (size_t)(c->n_recv_slots > 0 ? c->n_recv_slots : 1);
+    ok = ok && cudaMalloc(&c->d_recv_w1, per * n) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_recv_w3, per * n) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_recv_w2, per * n) == cudaSuccess;
+  }
   ok = ok && cudaMallocHost(&c->h_counts, sizeof(int32_t) * cfg->E) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_status, sizeof(uint32_t)) == cudaSuccess;
@@ -272,6 +321,9 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFree(c->d_home_groups);
   cudaFree(c->d_dyn_groups);
   cudaFree(c->d_mask);
+  cudaFree(c->d_recv_w1);
+  cudaFree(c->d_recv_w3);
+  cudaFree(c->d_recv_w2);
   cudaFreeHost(c->h_counts);
   cudaFreeHost(c->h_dyn_groups);
   cudaFreeHost(c->h_status);
@@ -371,6 +423,7 @@ static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void
   a.groups = groups; a.n_groups = n_groups; a.which = which;
   a.E = c->cfg.E; a.d = c->cfg.d; a.f = c->cfg.f; a.s_cap = (int64_t)c->s_cap;
   a.status = c->d_status; a.num_sms = c->num_sms; a.pair = pair;
+  a.recv_w1 = c->d_recv_w1; a.recv_w3 = c->d_recv_w3; a.recv_w2 = c->d_recv_w2; a.n_recv_slots = c->n_recv_slots;
   return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err));
 }
 
@@ -461,6 +514,7 @@ static int harvest_slot(feplb_ctx* c, int r) {
   t.dev_counts_to_static_start_us = el(ev[EV_COUNTS], ev[EV_STATIC0]);
   t.dev_counts_to_static_end_us = el(ev[EV_COUNTS], ev[EV_STATIC1]);
   t.dev_total_us = el(ev[EV_T0], ev[EV_COMBINE]);
+  t.dev_counts_to_copies_done_us = t.phase2_copy_bytes > 0 ? el(ev[EV_COUNTS], ev[EV_COPIES]) : 0.0;
   cudaGetLastError();
   const double* src = reinterpret_cast<const double*>(&t);
   double* dst = reinterpret_cast<double*>(&c->tl_sum);
@@ -500,6 +554,8 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   }
   c->t0 = clk::now();
   c->timeline_valid = true;
+  c->tl.phase2_copy_bytes = 0;
+  c->tl.dev_counts_to_copies_done_us = 0;
   TL_EVENT(EV_T0);
   // step 1: counts, rank loads, segment offsets and the home group table in two launches; the
   // planner thread starts as soon as the counts reach the host
@@ -518,6 +574,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
                                        rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
                                        (int64_t)c->s_cap, c->d_status, st, &c->launches));
+  c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
   if ((rc = feplb_plan_async(c, counts, dyn_mask_host, stream)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);

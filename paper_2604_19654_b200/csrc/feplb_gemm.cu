@@ -83,6 +83,7 @@ struct GemmParams {
   int n_tiles_n;        // N tiles per M tile
   int num_k_blocks;     // K / 64
   int b_rows_per_expert;  // rows of one expert in the B tensor maps
+  int n_recv_slots;     // slots of the receive buffer of migrated experts' weights (0 = none)
   int bn;               // rows of one B half tile (64 or 128); the MMA has N = 2*bn
   __nv_bfloat16* out;
   int ld_out;           // elements between output rows
@@ -256,7 +257,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 __device__ __forceinline__ float silu_f(float a) { return __fdividef(a, 1.f + __expf(-a)); }
 
-struct TileCoord { int row0, rows_valid, expert, nt; };
+struct TileCoord { int row0, rows_valid, expert, slot, nt; };   // slot >= 0: weights in that receive slot
 
 // tile -> (group, M tile, N tile); N tiles of one M tile are consecutive so that CTAs running at
 // the same time share the A rows and sweep one expert's weights together (both stay in L2).
@@ -272,7 +273,8 @@ __device__ __forceinline__ TileCoord tile_coord(const SmemTail* t, int n_groups,
   TileCoord c;
   c.row0 = t->g_row_start[lo] + local * kRows;
   c.rows_valid = min(kRows, t->g_rows[lo] - local * kRows);
-  c.expert = t->g_expert[lo];
+  c.expert = t->g_expert[lo] & 0xffff;
+  c.slot = (t->g_expert[lo] >> 16) - 1;
   c.nt = tile - mt * n_tiles_n;
   return c;
 }
@@ -294,7 +296,8 @@ __device__ __forceinline__ void convert_slice(const uint32_t (&a)[32], const uin
 template <bool SWIGLU, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
-               const __grid_constant__ CUtensorMap tm_b1, const GemmParams p) {
+               const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_r0,
+               const __grid_constant__ CUtensorMap tm_r1, const GemmParams p) {
   constexpr int kStages = Ring<PAIR>::kStages, kStageBytes = Ring<PAIR>::kStageBytes;
   constexpr int kTileRows = Ring<PAIR>::kTileRows;
   extern __shared__ uint8_t smem_raw[];
@@ -318,6 +321,8 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     prefetch_tmap(&tm_a);
     prefetch_tmap(&tm_b0);
     prefetch_tmap(&tm_b1);
+    prefetch_tmap(&tm_r0);
+    prefetch_tmap(&tm_r1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&tail->full[s]), 1);
       mbar_init(smem_u32(&tail->empty[s]), 1);
@@ -349,14 +354,15 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int tiles = 0;
     if (selected && gr.rows > 0) {
       const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 &&
-                      (int64_t)gr.row_start + gr.rows <= p.s_cap;
+                      (int64_t)gr.row_start + gr.rows <= p.s_cap && gr.is_dynamic - 2 < p.n_recv_slots;
       if (ok) tiles = (gr.rows + kTileRows - 1) / kTileRows;
       else atomicOr(p.status, FEPLB_ST_GROUP);
     }
     tail->prefix[g + 1] = tiles;   // turned into a prefix sum below
     tail->g_row_start[g] = gr.row_start;
     tail->g_rows[g] = gr.rows;
-    tail->g_expert[g] = gr.expert;
+    // expert id in the low half; receive slot + 1 in the high half (0 = weights at home)
+    tail->g_expert[g] = (gr.expert & 0xffff) | ((gr.is_dynamic >= 2 ? gr.is_dynamic - 1 : 0) << 16);
   }
   tc_fence_before();
   __syncthreads();
@@ -396,7 +402,10 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       bool ok = true;
       for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
         const TileCoord c = tile_coord<kTileRows>(tail, p.n_groups, p.n_tiles_n, tile);
-        const int brow0 = c.expert * p.b_rows_per_expert + (SWIGLU ? c.nt * p.bn : c.nt * 2 * p.bn);
+        // weights of a migrated expert come from its slot of the receive buffer
+        const CUtensorMap* mb0 = c.slot >= 0 ? &tm_r0 : &tm_b0;
+        const CUtensorMap* mb1 = c.slot >= 0 ? &tm_r1 : &tm_b1;
+        const int brow0 = (c.slot >= 0 ? c.slot : c.expert) * p.b_rows_per_expert + (SWIGLU ? c.nt * p.bn : c.nt * 2 * p.bn);
         const int brow1 = SWIGLU ? brow0 : brow0 + p.bn;
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
           if (!(ok = mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status))) break;
@@ -408,13 +417,13 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t full0 = map_to_cta(full, 0);
             if (cta_rank == 0) mbar_expect_tx(full, stage_tx);
             tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
-            if (cta_rank == 0) tma_load_2d_pair(sb, &tm_b0, full0, kb * BK, brow0);
-            else tma_load_2d_pair(sb, &tm_b1, full0, kb * BK, brow1);
+            if (cta_rank == 0) tma_load_2d_pair(sb, mb0, full0, kb * BK, brow0);
+            else tma_load_2d_pair(sb, mb1, full0, kb * BK, brow1);
           } else {
             mbar_expect_tx(full, stage_tx);
             tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
-            tma_load_2d(sb, &tm_b0, full, kb * BK, brow0);
-            tma_load_2d(sb + b_half_bytes, &tm_b1, full, kb * BK, brow1);
+            tma_load_2d(sb, mb0, full, kb * BK, brow0);
+            tma_load_2d(sb + b_half_bytes, mb1, full, kb * BK, brow1);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -574,8 +583,8 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
 }
 
 template <bool SWIGLU, bool PAIR>
-cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const GemmParams& p,
-                       int num_sms, cudaStream_t st) {
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tr0,
+                       const CUtensorMap& tr1, const GemmParams& p, int num_sms, cudaStream_t st) {
   static int grid = 0;   // per instantiation: set on first use
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads);
@@ -610,7 +619,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUte
     grid = g;
   }
   cfg.gridDim = dim3(grid);
-  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, p);
+  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, tr0, tr1, p);
 }
 
 }  // namespace
@@ -630,7 +639,17 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
     snprintf(err, errn, "cuTensorMapEncodeTiled failed (driver entry point missing or bad pointer/shape)");
     return FEPLB_E_CUDA;
   }
+  // receive buffer of migrated experts' weights, addressed by slot like the home weights by expert
+  CUtensorMap tm_r1 = tm_w1, tm_r3 = tm_w3, tm_r2 = tm_w2;
+  const bool has_recv = a.recv_w1 && a.recv_w3 && a.recv_w2 && a.n_recv_slots > 0;
+  if (has_recv && (!make_tmap(&tm_r1, a.recv_w1, (uint64_t)a.n_recv_slots * a.f, (uint64_t)a.d, bn1) ||
+                   !make_tmap(&tm_r3, a.recv_w3, (uint64_t)a.n_recv_slots * a.f, (uint64_t)a.d, bn1) ||
+                   !make_tmap(&tm_r2, a.recv_w2, (uint64_t)a.n_recv_slots * a.d, (uint64_t)a.f, bn2))) {
+    snprintf(err, errn, "cuTensorMapEncodeTiled failed for the receive buffer");
+    return FEPLB_E_CUDA;
+  }
   GemmParams p1;
+  p1.n_recv_slots = has_recv ? a.n_recv_slots : 0;
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
   p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1;
   p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status;
@@ -638,12 +657,12 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d;
 
-  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st)
-                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, p1, a.num_sms, st);
+  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st)
+                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st);
   ++*n_launch;
   if (e == cudaSuccess) {
-    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st)
-               : launch_one<false, false>(tm_h, tm_w2, tm_w2, p2, a.num_sms, st);
+    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, p2, a.num_sms, st)
+               : launch_one<false, false>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, p2, a.num_sms, st);
     ++*n_launch;
   }
   if (e != cudaSuccess) {

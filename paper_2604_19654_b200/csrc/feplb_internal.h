@@ -61,6 +61,8 @@ struct feplb_gemm_args {
   uint32_t* status;
   int num_sms;
   int pair;   // 1: clusters of two CTAs on 256-row tiles (cta_group::2); 0: one CTA per 128-row tile
+  // receive buffer of migrated experts' weights ([n_recv_slots, f, d] x2 and [n_recv_slots, d, f]); may be null
+  const void* recv_w1; const void* recv_w3; const void* recv_w2; int n_recv_slots;
 };
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);

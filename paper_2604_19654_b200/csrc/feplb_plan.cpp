@@ -19,6 +19,7 @@ int feplb_validate_config(const feplb_config* c) {
   if (c->policy != FEPLB_POLICY_LITERAL && c->policy != FEPLB_POLICY_FIRST_FIT) return FEPLB_E_INVALID;
   if (c->split != 0 && c->split != 1) return FEPLB_E_INVALID;
   if (c->mask_policy != FEPLB_MASK_GIVEN && c->mask_policy != FEPLB_MASK_REACTIVE) return FEPLB_E_INVALID;
+  if (c->phase2_copy != 0 && c->phase2_copy != 1) return FEPLB_E_INVALID;
   if ((int64_t)c->T * c->K + (int64_t)c->E * (c->row_align - 1) > INT32_MAX) return FEPLB_E_INVALID;
   return FEPLB_OK;
 }

@@ -24,7 +24,7 @@ FFN_ALL, FFN_STATIC, FFN_DYNAMIC = 0, 1, 2
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "T", "K", "E", "R", "d", "f", "dyn", "max_num_dyn", "tau", "ranks_per_domain", "policy",
-        "split", "split_granule", "row_align", "mask_policy")]
+        "split", "split_granule", "row_align", "mask_policy", "phase2_copy")]
 
 
 class Move(C.Structure):
@@ -46,7 +46,8 @@ class Timeline(C.Structure):
         "host_enqueue_static_done_us", "host_counts_ready_us", "host_plan_done_us",
         "host_upload_enqueued_us", "host_join_us", "host_return_us", "plan_us",
         "dev_hist_us", "dev_dispatch_us", "dev_static_ffn_us", "dev_dynamic_ffn_us", "dev_combine_us",
-        "dev_counts_to_static_start_us", "dev_counts_to_static_end_us", "dev_total_us")]
+        "dev_counts_to_static_start_us", "dev_counts_to_static_end_us", "dev_total_us",
+        "dev_counts_to_copies_done_us", "phase2_copy_bytes")]
 
 
 class FeplbError(RuntimeError):
@@ -104,9 +105,9 @@ def lib() -> C.CDLL:
 
 def make_config(T, K, E, R, d, f, dyn=4, max_num_dyn=8, tau=0, ranks_per_domain=0,
                 policy=POLICY_FIRST_FIT, split=0, split_granule=128, row_align=1,
-                mask_policy=MASK_REACTIVE) -> Config:
+                mask_policy=MASK_REACTIVE, phase2_copy=0) -> Config:
     return Config(T, K, E, R, d, f, dyn, max_num_dyn, tau, ranks_per_domain, policy, split,
-                  split_granule, row_align, mask_policy)
+                  split_granule, row_align, mask_policy, phase2_copy)
 
 
 def config_from_workload(w, **kw) -> Config:

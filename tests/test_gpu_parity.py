@@ -415,3 +415,56 @@ def test_pipelined_host_forward_matches_the_synchronous_one():
     with pytest.raises(F.FeplbError):
         case.ctx.host_wait(2)
     case.close()
+
+
+# ----------------------------------------------------------------------------- Phase-2 weight copies
+
+@pytest.mark.parametrize("name,kw", [("cfg1", {}), ("cfg2", {}), ("cfg4", {"split": 1})])
+def test_phase2_weight_copies_leave_the_output_unchanged(name, kw):
+    """With phase2_copy the weights of migrated experts really travel to a receive buffer and the
+    dynamic GEMM reads them there; the layer output must be bit-identical to the relabel-only path
+    (Section 2.2: same expert, identical weights)."""
+    torch = _torch()
+    w = W.get_workload(name)
+    if name != "cfg1":
+        w = w.with_(T=1024)
+    weights = W.gen_weights(w)
+    base = DeviceCase(w, mb=0, weights=weights, **kw)
+    p0 = base.ctx.moe_forward(base.d_x, base.d_ids, base.d_gates, base.d_w1, base.d_w3, base.d_w2, base.buf)
+    base.ctx.check_status()
+    out0 = F.bf16_bits(base.buf.out).copy()
+    case = DeviceCase(w, mb=0, weights=weights, phase2_copy=1, **kw)
+    case.ctx.set_timeline(True)
+    p1 = case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    case.ctx.check_status()
+    assert p1.moves == p0.moves and p1.groups == p0.groups and len(p1.moves) >= 1
+    assert np.array_equal(F.bf16_bits(case.buf.out), out0)
+    tl = case.ctx.get_timeline()
+    assert tl["phase2_copy_bytes"] == 3 * w.d * w.f * 2 * len(p1.moves)
+    assert tl["dev_counts_to_copies_done_us"] > 0
+
+    # the kernel reads a migrated piece's weights from its receive slot, not from the home arrays:
+    # recompute one moved group with ZERO home weights and the slot label -> same rows of y_perm
+    e, src, dst, rows = p1.moves[0]
+    slot = dst * case.cfg.max_num_dyn + 0                          # first move into dst takes its first slot
+    assert all(m[2] != dst for m in p1.moves[:0])
+    grp = [g for g in p1.groups if g[0] == e and g[3] == dst][0]
+    y_ref = case.buf.y_perm[grp[1]: grp[1] + grp[2]].clone()
+    zero1 = torch.zeros_like(case.d_w1)
+    zero2 = torch.zeros_like(case.d_w2)
+    case.buf.y_perm[grp[1]: grp[1] + grp[2]] = 7.0
+    d_groups = upload_groups([(e, grp[1], grp[2], dst, 2 + slot)])
+    case.ctx.expert_ffn(case.buf.x_perm, zero1, zero1, zero2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
+    case.ctx.check_status()
+    assert torch.equal(case.buf.y_perm[grp[1]: grp[1] + grp[2]].view(torch.int16), y_ref.view(torch.int16))
+    d_groups = upload_groups([(e, grp[1], grp[2], dst, 1)])        # labelled "home weights": zeros in, zeros out
+    case.ctx.expert_ffn(case.buf.x_perm, zero1, zero1, zero2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
+    torch.cuda.synchronize()
+    assert not case.buf.y_perm[grp[1]: grp[1] + grp[2]].float().abs().max().item()
+    # a slot beyond the receive buffer is reported, not dereferenced
+    d_groups = upload_groups([(e, grp[1], grp[2], dst, 2 + 10 ** 6)])
+    case.ctx.expert_ffn(case.buf.x_perm, zero1, zero1, zero2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
+    with pytest.raises(F.FeplbError):
+        case.ctx.check_status()
+    base.close()
+    case.close()
