@@ -3,7 +3,9 @@
 // computes the static experts) and the per-micro-batch orchestration.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <chrono>
+#include <climits>
 #include <condition_variable>
 #include <cstdarg>
 #include <cstdio>
@@ -54,6 +56,9 @@ struct feplb_ctx {
   feplb_group* h_dyn_groups = nullptr;
   uint32_t* h_status = nullptr;
   uint8_t* h_mask = nullptr;
+  int32_t* h_ready_flag = nullptr;   // pinned: sequence number of the forward whose counts are in h_counts
+  int32_t flag_seq = 0;
+  int32_t job_flag_seq = 0;          // 0: the job waits on ev_counts instead
 
   cudaStream_t copy_stream = nullptr;
   // pipelined host-buffer path: input and output copy streams and per-slot events
@@ -125,14 +130,21 @@ void planner_main(feplb_ctx* c) {
       c->job = JOB_RUNNING;
     }
     int rc = FEPLB_OK;
-    // bounded wait for the copy of the counts (no blocking driver call: poll the event)
+    // bounded wait for the counts: either the scan kernel writes them straight into pinned host
+    // memory and raises a sequence flag (whole-layer path), or a copy was enqueued and its event is
+    // polled (stand-alone feplb_plan_async); no blocking driver call either way
     const auto w0 = clk::now();
-    for (;;) {
-      cudaError_t q = cudaEventQuery(c->ev_counts);
-      if (q == cudaSuccess) break;
-      if (q != cudaErrorNotReady) { rc = FEPLB_E_CUDA; break; }
-      if (std::chrono::duration<double>(clk::now() - w0).count() > 2.0) { rc = FEPLB_E_TIMEOUT; break; }
+    for (uint32_t spin = 0;; ++spin) {
+      if (c->job_flag_seq) {
+        if (*(volatile int32_t*)c->h_ready_flag == c->job_flag_seq) break;
+      } else {
+        cudaError_t q = cudaEventQuery(c->ev_counts);
+        if (q == cudaSuccess) break;
+        if (q != cudaErrorNotReady) { rc = FEPLB_E_CUDA; break; }
+      }
+      if ((spin & 1023u) == 1023u && std::chrono::duration<double>(clk::now() - w0).count() > 2.0) { rc = FEPLB_E_TIMEOUT; break; }
     }
+    std::atomic_thread_fence(std::memory_order_acquire);
     c->tl.host_counts_ready_us = us_since(c->t0);
     if (rc == FEPLB_OK) {
       const feplb_config& cfg = c->cfg;
@@ -271,6 +283,8 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   ok = ok && cudaMallocHost(&c->h_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_status, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_mask, cfg->E) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_ready_flag, sizeof(int32_t)) == cudaSuccess;
+  if (ok) *c->h_ready_flag = 0;
   ok = ok && cudaMemset(c->d_status, 0, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -328,6 +342,7 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFreeHost(c->h_dyn_groups);
   cudaFreeHost(c->h_status);
   cudaFreeHost(c->h_mask);
+  cudaFreeHost(c->h_ready_flag);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->in_stream) cudaStreamDestroy(c->in_stream);
   if (c->out_stream) cudaStreamDestroy(c->out_stream);
@@ -462,6 +477,20 @@ extern "C" int feplb_plan_async(feplb_ctx* c, const int32_t* counts, const uint8
   {
     std::lock_guard<std::mutex> lk(c->mu);
     c->job_mask = dyn_mask_host;
+    c->job_flag_seq = 0;
+    c->job = JOB_PENDING;
+  }
+  c->cv.notify_all();
+  return FEPLB_OK;
+}
+
+// Whole-layer path: the counts of this forward arrive in h_counts with sequence number `seq`.
+static int plan_kick_flag(feplb_ctx* c, const uint8_t* dyn_mask_host, int32_t seq) {
+  {
+    std::lock_guard<std::mutex> lk(c->mu);
+    if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "moe_forward: a plan is already pending");
+    c->job_mask = dyn_mask_host;
+    c->job_flag_seq = seq;
     c->job = JOB_PENDING;
   }
   c->cv.notify_all();
@@ -571,11 +600,14 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     CUDA_TRY(c, cudaMemcpyAsync(c->d_mask, c->h_mask, g.E, cudaMemcpyHostToDevice, st));
     mask_dev = c->d_mask;
   }
+  c->flag_seq = c->flag_seq == INT32_MAX ? 1 : c->flag_seq + 1;
+  const int32_t seq = c->flag_seq;
   CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
                                        rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
-                                       (int64_t)c->s_cap, c->d_status, st, &c->launches));
+                                       (int64_t)c->s_cap, c->d_status, c->h_counts, c->h_ready_flag, seq, st,
+                                       &c->launches));
   c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
-  if ((rc = feplb_plan_async(c, counts, dyn_mask_host, stream)) != FEPLB_OK) return rc;
+  if ((rc = plan_kick_flag(c, dyn_mask_host, seq)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);
   // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move
@@ -585,7 +617,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
                                       (int64_t)c->s_cap, st, &c->launches);
     if (e == cudaSuccess)
       e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align, st,
-                              &c->launches, row_to_token);
+                              &c->launches, row_to_token, true);
     if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "dispatch launch: %s", cudaGetErrorString(e));
   }
   TL_EVENT(EV_DISPATCH);

@@ -37,13 +37,15 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
                                  cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
                                 const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token = nullptr);
+                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token = nullptr,
+                                bool programmatic = false);
 // Whole-layer path: histogram + one scan kernel that emits counts, rank loads, offsets, the home
 // group table and the -1 tail of row_to_token; then the ranking alone.
 cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R, int A, int dyn,
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                     int32_t* counts_host, int32_t* ready_flag_host, int32_t seq,
                                      cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
                               const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,

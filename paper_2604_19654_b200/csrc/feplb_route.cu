@@ -15,6 +15,30 @@
 
 namespace {
 
+// Programmatic dependent launch: a kernel launched with the attribute below may be scheduled
+// while the kernel before it in the stream drains; pdl_sync() holds it until that kernel's
+// results are complete (a no-op for ordinary launches) and lets its own successor do the same.
+__device__ __forceinline__ void pdl_sync() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, bool programmatic,
+                   Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = programmatic ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kChunks = FEPLB_SLOTS_PER_BLOCK / kThreads;   // 32-slot chunks per warp (4)
@@ -52,6 +76,7 @@ k_block_hist(const int32_t* __restrict__ ids, int64_t S, int E, int L, int32_t* 
   extern __shared__ int wh[];
   int id[kChunks];
   unsigned mk[kChunks];
+  pdl_sync();
   if (warp_histograms(ids, S, E, wh, id, mk)) atomicOr(status, FEPLB_ST_RANGE);
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += kThreads) {
@@ -126,11 +151,13 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
              const uint8_t* __restrict__ mask_in, int32_t* __restrict__ counts_out,
              int32_t* __restrict__ rank_load_out, int32_t* __restrict__ pad_off,
              feplb_group* __restrict__ groups, uint8_t* __restrict__ mask_out,
-             int32_t* __restrict__ row_to_token, int64_t s_cap) {
+             int32_t* __restrict__ row_to_token, int64_t s_cap,
+             int32_t* __restrict__ counts_host, volatile int32_t* ready_flag_host, int32_t seq) {
   __shared__ int tmp[64];
   __shared__ int sc[FEPLB_MAX_EXPERTS];
   const int e = threadIdx.x;
   int c = 0;
+  pdl_sync();
   if (e < E) {
     // exclusive scan over CTAs, eight independent loads in flight per round (the in-place stores
     // would otherwise serialise every load behind the previous store)
@@ -148,6 +175,10 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
     c = run;
     counts_out[e] = c;
     sc[e] = c;
+    if (counts_host) {           // straight into pinned host memory: the planner thread polls the flag
+      counts_host[e] = c;
+      __threadfence_system();
+    }
   }
   int total;
   const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, &total);   // also orders sc[] for all threads
@@ -171,6 +202,11 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
     for (int o = e * L; o < (e + 1) * L; ++o) sum += sc[o];
     rank_load_out[e] = sum;
   }
+  // (the scan's barriers above ordered every thread's host writes before this flag)
+  if (counts_host && e == 0) {
+    __threadfence_system();
+    *ready_flag_host = seq;
+  }
   for (int64_t i = (int64_t)total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
 }
 
@@ -182,6 +218,7 @@ k_rank(const int32_t* __restrict__ ids, int64_t S, int K, int E, const int32_t* 
   extern __shared__ int wh[];
   int id[kChunks];
   unsigned mk[kChunks];
+  pdl_sync();
   warp_histograms(ids, S, E, wh, id, mk);
   __syncthreads();
   // chain the warps: wh[w][e] becomes the first row of warp w's slots of expert e
@@ -229,6 +266,7 @@ constexpr int kGatherUnroll = 4;
 __global__ void __launch_bounds__(kThreads)
 k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, uint4* __restrict__ x_perm,
          int T, int K, int chunks) {
+  pdl_sync();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * kThreads) >> 5;
@@ -267,6 +305,7 @@ k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, u
 __global__ void __launch_bounds__(kThreads)
 k_zero_pad(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_off, uint4* __restrict__ x_perm,
            int chunks, int32_t* __restrict__ row_to_token) {
+  pdl_sync();
   const int e = blockIdx.x;
   const int64_t r0 = (int64_t)pad_off[e] + counts[e], r1 = pad_off[e + 1];
   if (row_to_token)
@@ -344,22 +383,21 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
 
 cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
                                 const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token) {
+                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token, bool programmatic) {
   cudaError_t err;
   const int chunks = d / 8;
   if (A > 1) {
-    k_zero_pad<<<E, kThreads, 0, st>>>(counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token);
+    err = launch(k_zero_pad, E, kThreads, 0, st, programmatic, counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token);
     ++*n_launch;
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    if (err != cudaSuccess) return err;
   }
   if (T == 0) return cudaSuccess;
   const int64_t units = (int64_t)T * ((chunks + 32 * kGatherUnroll - 1) / (32 * kGatherUnroll));
   int blocks = 148 * 8;   // 8 CTAs of 256 threads per SM are resident
   const int64_t need = (units + kWarps - 1) / kWarps;
   if (need < blocks) blocks = (int)need;
-  k_gather<<<blocks, kThreads, 0, st>>>((const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch(k_gather, blocks, kThreads, 0, st, programmatic, (const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
 }
 
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
@@ -373,18 +411,19 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                     int32_t* counts_host, int32_t* ready_flag_host, int32_t seq,
                                      cudaStream_t st, int64_t* n_launch) {
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   if (nb) {
-    k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E, block_hist, nullptr, nullptr, status);
+    err = launch(k_block_hist, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, E, E, block_hist,
+                 (int32_t*)nullptr, (int32_t*)nullptr, status);
     ++*n_launch;
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    if (err != cudaSuccess) return err;
   }
-  k_scan_fused<<<1, 1024, 0, st>>>(block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off, groups,
-                                   mask_out, row_to_token, s_cap);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch(k_scan_fused, 1, 1024, 0, st, true, block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off,
+                groups, mask_out, row_to_token, s_cap, counts_host, (volatile int32_t*)ready_flag_host, seq);
 }
 
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
@@ -392,7 +431,7 @@ cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const
                               cudaStream_t st, int64_t* n_launch) {
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   if (!nb) return cudaSuccess;
-  k_rank<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, K, E, block_base, pad_off, slot_to_row, row_to_token, s_cap);
   ++*n_launch;
-  return cudaGetLastError();
+  return launch(k_rank, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, K, E, block_base, pad_off, slot_to_row,
+                row_to_token, s_cap);
 }
