@@ -286,6 +286,15 @@ int feplb_get_timeline(feplb_ctx* ctx, feplb_timeline* out);
  * number.  The stage events of up to 16 forwards stay outstanding, so timing does not make the
  * host wait for the GPU between forwards; this call waits for the outstanding ones. */
 int feplb_timeline_totals(feplb_ctx* ctx, feplb_timeline* sum, int64_t* n_forwards, int32_t reset);
+/* Bound (milliseconds, default 2000) of the planner thread's wait for the counts.  When it expires
+ * the pending plan fails with FEPLB_E_TIMEOUT (returned by feplb_plan_wait / feplb_moe_forward) and
+ * the context stays usable.  Not allowed while a plan is pending. */
+int feplb_set_planner_timeout(feplb_ctx* ctx, int32_t timeout_ms);
+/* Self-test of the device-side bounded waits: launches one thread that waits, with the routine
+ * the GEMM kernels use, on an mbarrier nothing ever completes, limited to limit_us microseconds.
+ * Returns FEPLB_OK if the wait gave up, raised the status bit and the kernel returned normally;
+ * FEPLB_E_STATE otherwise.  The status word is clear afterwards.  Synchronises `stream`. */
+int feplb_selftest_bounded_wait(feplb_ctx* ctx, int32_t limit_us, void* stream);
 /* Number of kernels this library has launched on `ctx` since creation. */
 int64_t feplb_launch_count(const feplb_ctx* ctx);
 

@@ -59,6 +59,7 @@ struct feplb_ctx {
   int32_t* h_ready_flag = nullptr;   // pinned: sequence number of the forward whose counts are in h_counts
   int32_t flag_seq = 0;
   int32_t job_flag_seq = 0;          // 0: the job waits on ev_counts instead
+  int32_t planner_timeout_ms = 2000; // bound of the planner's wait for the counts
 
   cudaStream_t copy_stream = nullptr;
   // pipelined host-buffer path: input and output copy streams and per-slot events
@@ -142,7 +143,7 @@ void planner_main(feplb_ctx* c) {
         if (q == cudaSuccess) break;
         if (q != cudaErrorNotReady) { rc = FEPLB_E_CUDA; break; }
       }
-      if ((spin & 1023u) == 1023u && std::chrono::duration<double>(clk::now() - w0).count() > 2.0) { rc = FEPLB_E_TIMEOUT; break; }
+      if ((spin & 1023u) == 1023u && std::chrono::duration<double>(clk::now() - w0).count() > 1e-3 * c->planner_timeout_ms) { rc = FEPLB_E_TIMEOUT; break; }
     }
     std::atomic_thread_fence(std::memory_order_acquire);
     c->tl.host_counts_ready_us = us_since(c->t0);
@@ -630,7 +631,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   // join the planner (always, so that the context returns to idle), then step 5
   const feplb_group* dyn_groups = nullptr;
   int32_t n_dyn = 0;
-  int rc_join = feplb_plan_wait(c, 2000, plan_copy, &dyn_groups, &n_dyn, stream);
+  int rc_join = feplb_plan_wait(c, c->planner_timeout_ms + 500, plan_copy, &dyn_groups, &n_dyn, stream);
   c->tl.host_join_us = us_since(c->t0);
   if (rc != FEPLB_OK) return rc;
   if (rc_join != FEPLB_OK) return rc_join;
@@ -744,4 +745,28 @@ extern "C" int feplb_timeline_totals(feplb_ctx* c, feplb_timeline* sum, int64_t*
     c->tl_n = 0;
   }
   return FEPLB_OK;
+}
+
+extern "C" int feplb_set_planner_timeout(feplb_ctx* c, int32_t timeout_ms) {
+  if (!c || timeout_ms < 1) return FEPLB_E_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "set_planner_timeout: a plan is pending");
+  c->planner_timeout_ms = timeout_ms;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_selftest_bounded_wait(feplb_ctx* c, int32_t limit_us, void* stream) {
+  if (!c || limit_us < 1 || limit_us > 1000000) return FEPLB_E_INVALID;
+  cudaStream_t st = (cudaStream_t)stream;
+  int rc = feplb_check_status(c, stream);          // start from a clean status word
+  if (rc != FEPLB_OK) return rc;
+  int* d_flag = reinterpret_cast<int*>(c->d_pad_off);   // scratch word, rewritten by the next dispatch
+  CUDA_TRY(c, cudaMemsetAsync(d_flag, 0xFF, sizeof(int), st));
+  CUDA_TRY(c, feplb_launch_wait_selftest(c->d_status, 1000ull * limit_us, d_flag, st));
+  ++c->launches;
+  int gave_up = -1;
+  CUDA_TRY(c, cudaMemcpyAsync(&gave_up, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st));
+  rc = feplb_check_status(c, stream);              // synchronises; expected: FEPLB_E_DEVICE from the wait
+  if (rc == FEPLB_E_DEVICE && gave_up == 1) return FEPLB_OK;
+  return fail(c, FEPLB_E_STATE, "bounded-wait self-test: status %d, gave_up %d", rc, gave_up);
 }

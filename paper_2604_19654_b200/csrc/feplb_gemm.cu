@@ -119,7 +119,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 // Bounded wait.  Returns false if the CTA is aborting or the limit expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -128,7 +129,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const unsigned long long now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(status, FEPLB_ST_WAIT);
         return false;
@@ -551,6 +552,20 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing will ever complete.
+// The wait must give up after limit_ns, raise FEPLB_ST_WAIT and let the kernel return normally.
+__global__ void k_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    fence_barrier_init();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, limit_ns);
+    *gave_up = ok ? 0 : 1;
+  }
+}
+
 // ------------------------------------------------------------------------------------------ host
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -670,4 +685,9 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
     return FEPLB_E_CUDA;
   }
   return FEPLB_OK;
+}
+
+cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up, cudaStream_t st) {
+  k_wait_selftest<<<1, 32, 0, st>>>(status, limit_ns, gave_up);
+  return cudaGetLastError();
 }

@@ -67,6 +67,8 @@ struct feplb_gemm_args {
   const void* recv_w1; const void* recv_w3; const void* recv_w2; int n_recv_slots;
 };
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
+// One thread waits (bounded by limit_ns) on an mbarrier nobody completes; *gave_up = 1 and FEPLB_ST_WAIT expected.
+cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up, cudaStream_t st);
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
 #endif
 

@@ -94,6 +94,8 @@ def lib() -> C.CDLL:
             "feplb_set_timeline": (C.c_int, [vp, i32]),
             "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
             "feplb_timeline_totals": (C.c_int, [vp, C.POINTER(Timeline), C.POINTER(i64), i32]),
+            "feplb_set_planner_timeout": (C.c_int, [vp, i32]),
+            "feplb_selftest_bounded_wait": (C.c_int, [vp, i32, vp]),
             "feplb_launch_count": (i64, [vp]),
         }
         for name, (res, args) in sig.items():
@@ -325,6 +327,14 @@ class Context:
         t, n = Timeline(), C.c_int64()
         self._chk(lib().feplb_timeline_totals(self._h, C.byref(t), C.byref(n), int(bool(reset))), "feplb_timeline_totals")
         return {k: getattr(t, k) for k, _ in Timeline._fields_}, n.value
+
+    def set_planner_timeout(self, timeout_ms: int):
+        self._chk(lib().feplb_set_planner_timeout(self._h, int(timeout_ms)), "feplb_set_planner_timeout")
+
+    def selftest_bounded_wait(self, limit_us=2000, stream=None):
+        """Raises unless a device-side wait on a barrier nobody completes gives up after limit_us."""
+        self._chk(lib().feplb_selftest_bounded_wait(self._h, int(limit_us), self._stream(stream)),
+                  "feplb_selftest_bounded_wait")
 
     def launch_count(self) -> int:
         return int(lib().feplb_launch_count(self._h))

@@ -468,3 +468,34 @@ def test_phase2_weight_copies_leave_the_output_unchanged(name, kw):
         case.ctx.check_status()
     base.close()
     case.close()
+
+
+# ----------------------------------------------------------------------------- bounded waits, no GPU hang
+
+def test_device_wait_gives_up_and_reports():
+    """A device-side wait on a barrier that nothing completes ends after its limit with a status
+    bit and a normal kernel return; the context keeps working afterwards."""
+    case = DeviceCase(W.get_workload("cfg1"))
+    case.ctx.selftest_bounded_wait(limit_us=3000)
+    case.ctx.check_status()                                            # clean again
+    _check_forward(case)
+    case.close()
+
+
+def test_planner_times_out_when_the_counts_do_not_arrive_and_recovers():
+    """The counts are withheld by keeping the stream busy with other work; the planner's bounded
+    wait expires (FEPLB_E_TIMEOUT), nothing hangs, and the next forward succeeds."""
+    torch = _torch()
+    case = DeviceCase(W.get_workload("cfg1"))
+    case.ctx.set_planner_timeout(5)                                    # 5 ms
+    a = torch.randn(8192, 8192, device="cuda", dtype=torch.bfloat16)
+    for _ in range(60):                                                # ~60 x 0.8 ms of matmuls ahead of the layer
+        a @ a
+    with pytest.raises(F.FeplbError) as ei:
+        case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    assert ei.value.code == F.E_TIMEOUT
+    torch.cuda.synchronize()
+    case.ctx.set_planner_timeout(2000)
+    case.ctx.check_status()
+    _check_forward(case)
+    case.close()
