@@ -159,7 +159,24 @@ int feplb_select_dynamic(const int64_t* score, int32_t E, int32_t R, int32_t dyn
  * per-rank loads.  Returns FEPLB_E_NOMEM if a capacity is too small.  Pure function. */
 int feplb_plan(const feplb_config* cfg, const int32_t* counts, const uint8_t* dyn_mask, feplb_plan_out* out);
 
+/* Macro level (Section 2.3: a Router Predictor re-places experts from historical routing
+ * statistics at checkpoint time; the paper gives no algorithm).  feplb_ema_update keeps the
+ * statistics: ema[e] <- decay*ema[e] + (1-decay)*counts[e] (host arrays of E entries).
+ * feplb_place_experts assigns experts to ranks by the capacity-constrained longest-processing-time
+ * greedy: experts by descending load (ties to the lower id), each to the least loaded rank that
+ * still has room for one of its E/R experts (ties to the lower rank).  new_index[e] (host, E
+ * entries) is the position expert e moves to; its new home rank is new_index[e] / (E/R).  The
+ * caller permutes the weights and maps router ids through new_index. */
+int feplb_ema_update(double* ema, const int32_t* counts, int32_t E, double decay);
+int feplb_place_experts(const double* load, int32_t E, int32_t R, int32_t* new_index);
+
 /* ---- device steps ------------------------------------------------------------------------- */
+
+/* Step 0, optional (Section 2.3: "the router produces routing decisions"; Section 3.1: top-k
+ * routing): top-k gating from router logits.  Per token the K largest of its E logits in
+ * descending order, ties to the lower expert id; gates = softmax over the K selected logits
+ * (fp32).  logits dev float [T,E] (finite values) -> topk_ids dev int32 [T,K], gates dev float [T,K]. */
+int feplb_route_topk(feplb_ctx* ctx, const float* logits, int32_t* topk_ids, float* gates, void* stream);
 
 /* Step 1 (Section 2.2: per-expert token counts after Phase 1).
  * topk_ids dev int32 [T,K] -> counts dev int32 [E], rank_load dev int32 [R] (both overwritten).

@@ -37,6 +37,13 @@ combine         "Combine phase returns results" (Section 2.3) = gate-weighted su
                 scalar loops
 token_straggler the paper's metric max_d T_d - mean (Section 3.1 "Metrics").  pinned: Table 3
                 arithmetic
+route_topk      top-k gating of the router (Sections 2.3, 3.1); gates = softmax over the selected
+                logits is the workloads' definition, not the paper's.  PARITY UNPINNED against
+                the paper; pinned: library stable sort, closed forms (sigmoid, plain softmax)
+place_experts   macro-level expert-to-device assignment from historical load (Section 2.3, Router
+                Predictor; no algorithm given): capacity-constrained LPT greedy, a reading.
+                PARITY UNPINNED against the paper; pinned: permutation invariant, brute-force
+                optimum and the 4/3 LPT bound on tiny inputs
 """
 from __future__ import annotations
 
@@ -352,3 +359,54 @@ def moe_layer(x_bits, topk_ids, gates, w1_bits, w3_bits, w2_bits, E: int, A: int
     y = expert_ffn(x_rows, sub_ids.reshape(-1), w1_bits, w3_bits, w2_bits)
     s2r = np.arange(tokens.shape[0] * K).reshape(-1, K)
     return combine(y, s2r, np.asarray(gates)[tokens])
+
+
+# ----------------------------------------------------------------------------- router, placement
+
+def route_topk(logits: np.ndarray, K: int):
+    """Top-k gating (Section 2.3: "the router produces routing decisions"; Section 3.1: top-k
+    routing, no auxiliary loss): per token the K largest logits in descending order, ties to the
+    lower expert id; gates = softmax over the K selected logits.  The paper gives no formula for
+    the gates; softmax over the selected logits is the workloads' definition.  PARITY UNPINNED
+    against the paper; pinned against a library sort and closed forms.
+    Returns (topk_ids int64 [T,K], gates float64 [T,K]).
+    """
+    z = np.asarray(logits, np.float64)
+    T, E = z.shape
+    ids = np.empty((T, K), np.int64)
+    gates = np.empty((T, K), np.float64)
+    for t in range(T):
+        order = sorted(range(E), key=lambda e: (-z[t, e], e))[:K]
+        sel = np.array([z[t, e] for e in order])
+        w = np.exp(sel - sel.max())
+        ids[t] = order
+        gates[t] = w / w.sum()
+    return ids, gates
+
+
+def ema_update(ema, counts, decay: float):
+    """Historical routing statistics of the macro level (Section 2.3): ema <- decay*ema + (1-decay)*counts."""
+    return decay * np.asarray(ema, np.float64) + (1.0 - decay) * np.asarray(counts, np.float64)
+
+
+def place_experts(load, R: int) -> np.ndarray:
+    """Expert-to-device assignment from historical load (Section 2.3, Router Predictor; the paper
+    gives no algorithm).  Reading: longest-processing-time greedy under the capacity of L = E/R
+    experts per rank -- experts by descending load (ties -> lower id), each to the least loaded
+    rank that still has room (ties -> lower rank).  PARITY UNPINNED against the paper.
+    Returns new_index int64 [E]: expert e moves to position new_index[e] (rank = position // L).
+    """
+    load = [float(v) for v in np.asarray(load).tolist()]
+    E = len(load)
+    assert E % R == 0
+    L = E // R
+    order = sorted(range(E), key=lambda e: (-load[e], e))
+    rank_load = [0.0] * R
+    fill = [0] * R
+    new_index = [0] * E
+    for e in order:
+        r = min((r for r in range(R) if fill[r] < L), key=lambda r: (rank_load[r], r))
+        new_index[e] = r * L + fill[r]
+        fill[r] += 1
+        rank_load[r] += load[e]
+    return np.array(new_index, np.int64)

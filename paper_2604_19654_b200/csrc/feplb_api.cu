@@ -770,3 +770,12 @@ extern "C" int feplb_selftest_bounded_wait(feplb_ctx* c, int32_t limit_us, void*
   if (rc == FEPLB_E_DEVICE && gave_up == 1) return FEPLB_OK;
   return fail(c, FEPLB_E_STATE, "bounded-wait self-test: status %d, gave_up %d", rc, gave_up);
 }
+
+extern "C" int feplb_route_topk(feplb_ctx* c, const float* logits, int32_t* topk_ids, float* gates, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (c->cfg.K > c->cfg.E) return fail(c, FEPLB_E_INVALID, "route_topk: K > E");
+  if (c->cfg.T > 0 && (!logits || !topk_ids || !gates)) return fail(c, FEPLB_E_INVALID, "route_topk: null pointer");
+  CUDA_TRY(c, feplb_launch_route_topk(logits, c->cfg.T, c->cfg.E, c->cfg.K, topk_ids, gates, (cudaStream_t)stream,
+                                      &c->launches));
+  return FEPLB_OK;
+}

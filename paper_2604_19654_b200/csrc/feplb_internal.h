@@ -55,6 +55,9 @@ cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_
 cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row, const float* gates, void* out,
                                  int T, int K, int d, int num_sms, cudaStream_t st, int64_t* n_launch);
 
+cudaError_t feplb_launch_route_topk(const float* logits, int T, int E, int K, int32_t* ids, float* gates,
+                                    cudaStream_t st, int64_t* n_launch);
+
 struct feplb_gemm_args {
   const void* x_perm; const void* w1; const void* w3; const void* w2;
   void* h; void* y;

@@ -139,3 +139,29 @@ extern "C" int feplb_plan(const feplb_config* cfg, const int32_t* counts, const 
   out->n_groups = n_groups;
   return FEPLB_OK;
 }
+
+extern "C" int feplb_ema_update(double* ema, const int32_t* counts, int32_t E, double decay) {
+  if (!ema || !counts || E < 1 || !(decay >= 0.0 && decay <= 1.0)) return FEPLB_E_INVALID;
+  for (int e = 0; e < E; ++e) ema[e] = decay * ema[e] + (1.0 - decay) * (double)counts[e];
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_place_experts(const double* load, int32_t E, int32_t R, int32_t* new_index) {
+  if (!load || !new_index || E < 1 || R < 1 || E % R) return FEPLB_E_INVALID;
+  const int L = E / R;
+  std::vector<int> order(E);
+  for (int e = 0; e < E; ++e) order[e] = e;
+  // heaviest first, lower id on ties
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return load[a] > load[b]; });
+  std::vector<double> rank_load(R, 0.0);
+  std::vector<int> fill(R, 0);
+  for (int e : order) {
+    int best = -1;   // least loaded rank with room, lowest id on ties
+    for (int r = 0; r < R; ++r)
+      if (fill[r] < L && (best < 0 || rank_load[r] < rank_load[best])) best = r;
+    new_index[e] = best * L + fill[best];
+    fill[best] += 1;
+    rank_load[best] += load[e];
+  }
+  return FEPLB_OK;
+}

@@ -341,6 +341,55 @@ k_home_groups(const int32_t* __restrict__ counts, const uint8_t* __restrict__ ma
   if (mask_out) mask_out[e] = (uint8_t)is_dyn;
 }
 
+// Router top-k gating (paper Sections 2.3 and 3.1: top-k routing, no auxiliary loss): one warp per
+// token.  Lane l holds logits l, l+32, ...; K rounds of a warp arg-max (larger value, then lower
+// expert id) pick the experts in descending order; gates = softmax over the K selected logits.
+template <int NPER>
+__global__ void __launch_bounds__(kThreads)
+k_route_topk(const float* __restrict__ logits, int T, int E, int K, int32_t* __restrict__ ids,
+             float* __restrict__ gates) {
+  const int lane = threadIdx.x & 31;
+  const int warp = (blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int nwarps = (gridDim.x * kThreads) >> 5;
+  for (int t = warp; t < T; t += nwarps) {
+    float v[NPER];
+#pragma unroll
+    for (int i = 0; i < NPER; ++i) {
+      const int e = i * 32 + lane;
+      v[i] = e < E ? logits[(int64_t)t * E + e] : -INFINITY;
+    }
+    unsigned taken = 0;
+    float sel_val = 0.f;
+    int sel_idx = 0;
+    for (int k = 0; k < K; ++k) {
+      float best = -INFINITY;
+      int bidx = 0x7fffffff;
+#pragma unroll
+      for (int i = 0; i < NPER; ++i) {
+        const int e = i * 32 + lane;
+        if (e < E && !((taken >> i) & 1u) && (v[i] > best || bidx == 0x7fffffff)) { best = v[i]; bidx = e; }
+      }
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bidx, o);
+        if (oi != 0x7fffffff && (bidx == 0x7fffffff || ov > best || (ov == best && oi < bidx))) { best = ov; bidx = oi; }
+      }
+      if ((bidx & 31) == lane) taken |= 1u << (bidx >> 5);
+      if (lane == k) { sel_val = best; sel_idx = bidx; }
+    }
+    const float m = __shfl_sync(0xffffffffu, sel_val, 0);       // the first pick is the maximum
+    float ex = lane < K ? expf(sel_val - m) : 0.f;
+    float sum = ex;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane < K) {
+      ids[(int64_t)t * K + lane] = sel_idx;
+      gates[(int64_t)t * K + lane] = ex / sum;
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t feplb_launch_block_hist(const int32_t* ids, int64_t S, int E, int R, int32_t* block_hist,
@@ -434,4 +483,20 @@ cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const
   ++*n_launch;
   return launch(k_rank, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, K, E, block_base, pad_off, slot_to_row,
                 row_to_token, s_cap);
+}
+
+cudaError_t feplb_launch_route_topk(const float* logits, int T, int E, int K, int32_t* ids, float* gates,
+                                    cudaStream_t st, int64_t* n_launch) {
+  if (T == 0) return cudaSuccess;
+  int blocks = (T + kWarps - 1) / kWarps;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  const int nper = (E + 31) / 32;
+  ++*n_launch;
+  if (nper <= 1) k_route_topk<1><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  else if (nper <= 2) k_route_topk<2><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  else if (nper <= 4) k_route_topk<4><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  else if (nper <= 8) k_route_topk<8><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  else if (nper <= 16) k_route_topk<16><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  else k_route_topk<32><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);
+  return cudaGetLastError();
 }

@@ -79,6 +79,9 @@ def lib() -> C.CDLL:
             "feplb_s_pad": (C.c_size_t, [C.POINTER(Config)]),
             "feplb_select_dynamic": (C.c_int, [C.POINTER(i64), i32, i32, i32, C.POINTER(C.c_uint8)]),
             "feplb_plan": (C.c_int, [C.POINTER(Config), C.POINTER(i32), C.POINTER(C.c_uint8), C.POINTER(PlanOut)]),
+            "feplb_ema_update": (C.c_int, [C.POINTER(C.c_double), C.POINTER(i32), i32, C.c_double]),
+            "feplb_place_experts": (C.c_int, [C.POINTER(C.c_double), i32, i32, C.POINTER(i32)]),
+            "feplb_route_topk": (C.c_int, [vp, vp, vp, vp, vp]),
             "feplb_route_hist": (C.c_int, [vp, vp, vp, vp, vp]),
             "feplb_dispatch": (C.c_int, [vp] * 8),
             "feplb_dispatch_noalloc": (C.c_int, [C.POINTER(Config)] + [vp] * 8),
@@ -158,6 +161,28 @@ def select_dynamic(score: Sequence[int], E: int, R: int, dyn: int) -> np.ndarray
                                     out.ctypes.data_as(C.POINTER(C.c_uint8)))
     if rc:
         raise FeplbError(rc, "feplb_select_dynamic")
+    return out
+
+
+def ema_update(ema: np.ndarray, counts, decay: float) -> np.ndarray:
+    """In place: ema <- decay*ema + (1-decay)*counts (float64 [E])."""
+    cnt = np.ascontiguousarray(counts, np.int32)
+    assert ema.dtype == np.float64 and ema.flags.c_contiguous and ema.shape == cnt.shape
+    rc = lib().feplb_ema_update(ema.ctypes.data_as(C.POINTER(C.c_double)), cnt.ctypes.data_as(C.POINTER(C.c_int32)),
+                                cnt.shape[0], float(decay))
+    if rc:
+        raise FeplbError(rc, "feplb_ema_update")
+    return ema
+
+
+def place_experts(load, R: int) -> np.ndarray:
+    """Macro-level placement: new_index[e] = position expert e moves to (host only)."""
+    ld = np.ascontiguousarray(load, np.float64)
+    out = np.zeros(ld.shape[0], np.int32)
+    rc = lib().feplb_place_experts(ld.ctypes.data_as(C.POINTER(C.c_double)), ld.shape[0], int(R),
+                                   out.ctypes.data_as(C.POINTER(C.c_int32)))
+    if rc:
+        raise FeplbError(rc, "feplb_place_experts")
     return out
 
 
@@ -241,6 +266,10 @@ class Context:
 
     def check_status(self, stream=None):
         self._chk(lib().feplb_check_status(self._h, self._stream(stream)), "feplb_check_status")
+
+    def route_topk(self, logits, topk_ids, gates, stream=None):
+        self._chk(lib().feplb_route_topk(self._h, _ptr(logits), _ptr(topk_ids), _ptr(gates), self._stream(stream)),
+                  "feplb_route_topk")
 
     def route_hist(self, topk_ids, counts, rank_load, stream=None):
         self._chk(lib().feplb_route_hist(self._h, _ptr(topk_ids), _ptr(counts), _ptr(rank_load),

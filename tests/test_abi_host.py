@@ -124,3 +124,43 @@ def test_plan_capacity_error():
     rc = F.lib().feplb_plan(C.byref(cfg), cnt.ctypes.data_as(C.POINTER(C.c_int32)),
                             msk.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(p.c))
     assert rc == F.E_NOMEM
+
+
+@settings(max_examples=100, deadline=None)
+@given(st.sampled_from([(1, 4), (2, 2), (2, 8), (4, 4), (8, 16)]), st.integers(0, 2 ** 31), st.booleans())
+def test_place_experts_and_ema_match_oracle(shape, seed, ties):
+    R, L = shape
+    rng = np.random.default_rng(seed)
+    load = rng.integers(0, 5 if ties else 10 ** 6, size=R * L).astype(np.float64)
+    assert np.array_equal(F.place_experts(load, R), O.place_experts(load, R))
+    ema = rng.random(R * L)
+    counts = rng.integers(0, 1000, size=R * L)
+    ref = O.ema_update(ema, counts, 0.9)
+    assert np.array_equal(F.ema_update(ema.copy(), counts, 0.9), ref)
+
+
+def test_placement_lowers_the_straggler_of_drifting_routing():
+    """Macro level + micro level together on a synthetic drift: popularity = persistent part +
+    per-micro-batch noise.  Placing experts from the EMA of past counts lowers the unbalanced
+    straggler, and the per-micro-batch plan lowers it further."""
+    w = W.get_workload("cfg3")
+    rng = np.random.default_rng(4)
+    persistent = rng.dirichlet(np.full(w.E, 0.3))
+    ema = np.zeros(w.E)
+    def counts_of(mb):
+        p = 0.7 * persistent + 0.3 * np.random.default_rng(100 + mb).dirichlet(np.full(w.E, 0.3))
+        return np.random.default_rng(200 + mb).multinomial(w.S, p).astype(np.int32)
+    for mb in range(20):
+        F.ema_update(ema, counts_of(mb), 0.9)
+    pos = F.place_experts(ema, w.R)
+    inv = np.argsort(pos)                                       # expert sitting at each new position
+    before, placed, planned = [], [], []
+    for mb in range(20, 28):
+        c = counts_of(mb)
+        cp = c[inv]                                             # counts in the new expert order
+        before.append(O.straggler_ratio(c.reshape(w.R, w.L).sum(1)))
+        placed.append(O.straggler_ratio(cp.reshape(w.R, w.L).sum(1)))
+        p = F.plan(F.config_from_workload(w), cp, F.select_dynamic(cp, w.E, w.R, w.dyn))
+        planned.append(O.straggler_ratio(p.load_after))
+    assert np.mean(placed) < np.mean(before) and np.mean(planned) < np.mean(placed)
+    assert np.mean(planned) < 1.1

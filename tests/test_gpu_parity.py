@@ -499,3 +499,45 @@ def test_planner_times_out_when_the_counts_do_not_arrive_and_recovers():
     case.ctx.check_status()
     _check_forward(case)
     case.close()
+
+
+# ----------------------------------------------------------------------------- router top-k
+
+@pytest.mark.parametrize("T,E,K", [(1, 8, 2), (300, 8, 8), (1000, 64, 6), (513, 128, 8), (64, 1024, 32), (77, 48, 1)])
+def test_route_topk_parity(T, E, K):
+    """ids bit-exact (descending logit, ties to the lower id), gates within fp32 rounding of the
+    fp64 softmax over the selected logits."""
+    torch = _torch()
+    rng = np.random.default_rng(T + E + K)
+    logits = rng.standard_normal((T, E)).astype(np.float32)
+    if T > 2:
+        logits[1, :] = 0.5                                             # all tied
+        logits[2, E // 2] = logits[2, 0] = logits[2].max() + 1.0       # a tie at the top
+    w = _tiny(T, K, E, 1)
+    ctx = F.Context(F.config_from_workload(w))
+    ids = torch.zeros(T, K, dtype=torch.int32, device="cuda")
+    gates = torch.zeros(T, K, dtype=torch.float32, device="cuda")
+    ctx.route_topk(torch.from_numpy(logits).cuda(), ids, gates)
+    ctx.check_status()
+    ref_ids, ref_gates = O.route_topk(logits, K)
+    assert np.array_equal(ids.cpu().numpy(), ref_ids)
+    assert np.allclose(gates.cpu().numpy(), ref_gates, rtol=2e-6, atol=1e-7)
+    ctx.close()
+
+
+def test_router_feeds_the_layer():
+    """logits -> feplb_route_topk -> feplb_moe_forward equals the oracle run from the same logits."""
+    torch = _torch()
+    w = W.get_workload("cfg1")
+    rng = np.random.default_rng(3)
+    logits = (rng.standard_normal((w.T, w.E)) * 2).astype(np.float32)
+    case = DeviceCase(w)
+    d_ids = torch.zeros(w.T, w.K, dtype=torch.int32, device="cuda")
+    d_gates = torch.zeros(w.T, w.K, dtype=torch.float32, device="cuda")
+    case.ctx.route_topk(torch.from_numpy(logits).cuda(), d_ids, d_gates)
+    case.ctx.moe_forward(case.d_x, d_ids, d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    case.ctx.check_status()
+    ids, gates = O.route_topk(logits, w.K)
+    ref = O.moe_layer(case.x, ids, gates, case.w1, case.w3, case.w2, w.E)
+    assert_close(W.bf16_bits_to_f64(F.bf16_bits(case.buf.out)), ref, "router + layer")
+    case.close()

@@ -440,3 +440,50 @@ def test_staged_pipeline_equals_layer_definition():
         assert np.allclose(out, ref, rtol=1e-12, atol=1e-18)
     sub = np.array([0, 17, 255])
     assert np.allclose(O.moe_layer(x, ids, gates, w1, w3, w2, w.E, tokens=sub), ref[sub], rtol=1e-12, atol=1e-18)
+
+
+# ----------------------------------------------------------------------------- router, placement
+
+def test_route_topk_against_library_sort_and_closed_forms():
+    rng = np.random.default_rng(9)
+    z = rng.standard_normal((40, 12)).astype(np.float32)
+    z[3, 5] = z[3, 2]                                          # a tie: the lower id wins
+    z[7, :] = 0.25                                             # all equal: ids 0..K-1, uniform gates
+    ids, gates = O.route_topk(z, 4)
+    order = np.argsort(-z.astype(np.float64), axis=1, kind="stable")[:, :4]   # library stable sort
+    assert np.array_equal(ids, order)
+    assert ids[7].tolist() == [0, 1, 2, 3] and np.allclose(gates[7], 0.25)
+    assert np.allclose(gates.sum(1), 1.0) and np.all(np.diff(gates, axis=1) <= 1e-15)
+    # two selected logits a > b: gate = sigmoid(a - b)
+    ids2, g2 = O.route_topk(np.array([[1.0, 3.0, -2.0]]), 2)
+    assert ids2.tolist() == [[1, 0]] and g2[0, 0] == pytest.approx(1.0 / (1.0 + math.exp(-2.0)))
+    # K = E: plain softmax in sorted order
+    ids3, g3 = O.route_topk(z[:5], 12)
+    sm = np.exp(z[:5].astype(np.float64))
+    sm /= sm.sum(1, keepdims=True)
+    assert np.allclose(g3, np.take_along_axis(sm, ids3, axis=1))
+    # the workloads' generator is this router applied to its logits: same ids, same gates
+    w = W.get_workload("cfg1")
+    gen_ids, gen_gates = W.gen_routing(w, 0)
+    assert gen_ids.shape == (w.T, w.K) and np.allclose(gen_gates.sum(1), 1.0, atol=1e-6)
+
+
+def test_place_experts_invariants_and_bruteforce():
+    rng = np.random.default_rng(2)
+    for R, L in ((2, 2), (2, 3), (3, 2), (4, 4)):
+        load = rng.integers(1, 100, size=R * L).astype(float)
+        pos = O.place_experts(load, R)
+        assert sorted(pos.tolist()) == list(range(R * L))      # a permutation: every rank gets L experts
+        rl = np.zeros(R)
+        for e, p in enumerate(pos):
+            rl[p // L] += load[e]
+        if R * L <= 6:                                         # brute force: optimum over all balanced assignments
+            best = min(max(sum(load[e] for e in range(R * L) if a[e] == r) for r in range(R))
+                       for a in itertools.product(range(R), repeat=R * L)
+                       if all(a.count(r) == L for r in range(R)))
+            assert best <= rl.max() <= best * 4.0 / 3.0 + 1e-9  # the classical LPT bound
+    # equal loads -> round-robin placement; one heavy expert ends up with the lightest companions
+    assert O.place_experts([5, 5, 5, 5], 2).tolist() == [0, 2, 1, 3]
+    pos = O.place_experts([100, 1, 2, 3], 2)
+    assert pos[0] // 2 != pos[3] // 2 and pos[0] // 2 == pos[1] // 2   # 100 shares a rank with the lightest
+    assert np.allclose(O.ema_update([10.0, 0.0], [0.0, 10.0], 0.9), [9.0, 1.0])
