@@ -44,6 +44,10 @@ place_experts   macro-level expert-to-device assignment from historical load (Se
                 Predictor; no algorithm given): capacity-constrained LPT greedy, a reading.
                 PARITY UNPINNED against the paper; pinned: permutation invariant, brute-force
                 optimum and the 4/3 LPT bound on tiny inputs
+moe_layer_backward  gradients of the layer w.r.t. x, gates and the expert weights (Table 2 reports
+                backward times; the pass itself is not described): the chain rule of the forward
+                definition.                                               pinned: central finite
+                differences of the forward definition
 """
 from __future__ import annotations
 
@@ -410,3 +414,53 @@ def place_experts(load, R: int) -> np.ndarray:
         fill[r] += 1
         rank_load[r] += load[e]
     return np.array(new_index, np.int64)
+
+
+# ----------------------------------------------------------------------------- backward pass
+
+def dsilu(z: np.ndarray) -> np.ndarray:
+    """d/dz [z * sigmoid(z)] = sigmoid(z) * (1 + z * (1 - sigmoid(z)))."""
+    sg = 1.0 / (1.0 + np.exp(-z))
+    return sg * (1.0 + z * (1.0 - sg))
+
+
+def moe_layer_backward(x_bits, topk_ids, gates, w1_bits, w3_bits, w2_bits, d_out, E: int):
+    """Gradients of out[t,:] = sum_k gates[t,k] * FFN_{e(t,k)}(x[t,:]) (the layer of moe_layer)
+    with respect to x, gates and the expert weights, for the upstream gradient d_out [T,d]; all
+    fp64, the chain rule written out per (token, k) slot grouped by expert.  The paper reports
+    forward/backward layer times (Table 2) but does not describe the backward pass; this is the
+    plain derivative of the forward definition.  Pinned by central finite differences.
+    Returns (dx [T,d], dgates [T,K], dw1 [E,f,d], dw3 [E,f,d], dw2 [E,d,f]) in the weights' layout.
+    """
+    ids = np.asarray(topk_ids)
+    T, K = ids.shape
+    X = bf16_bits_to_f64(x_bits)
+    G = np.asarray(gates, np.float64)
+    dO = np.asarray(d_out, np.float64)
+    dx = np.zeros_like(X)
+    dg = np.zeros((T, K), np.float64)
+    dw1 = np.zeros(w1_bits.shape, np.float64)
+    dw3 = np.zeros(w3_bits.shape, np.float64)
+    dw2 = np.zeros(w2_bits.shape, np.float64)
+    for e in range(E):
+        tt, kk = np.nonzero(ids == e)
+        if tt.size == 0:
+            continue
+        W1 = bf16_bits_to_f64(w1_bits[e])      # [f, d]
+        W3 = bf16_bits_to_f64(w3_bits[e])
+        W2 = bf16_bits_to_f64(w2_bits[e])      # [d, f]
+        Xe = X[tt]
+        a = Xe @ W1.T
+        b = Xe @ W3.T
+        h = silu(a) * b
+        y = h @ W2.T
+        dy = G[tt, kk][:, None] * dO[tt]       # out = sum_k g * y
+        dg[tt, kk] = np.sum(dO[tt] * y, axis=1)
+        dh = dy @ W2
+        dw2[e] = dy.T @ h
+        da = dh * b * dsilu(a)
+        db = dh * silu(a)
+        dw1[e] = da.T @ Xe
+        dw3[e] = db.T @ Xe
+        np.add.at(dx, tt, da @ W1 + db @ W3)
+    return dx, dg, dw1, dw3, dw2

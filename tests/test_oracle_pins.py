@@ -487,3 +487,44 @@ def test_place_experts_invariants_and_bruteforce():
     pos = O.place_experts([100, 1, 2, 3], 2)
     assert pos[0] // 2 != pos[3] // 2 and pos[0] // 2 == pos[1] // 2   # 100 shares a rank with the lightest
     assert np.allclose(O.ema_update([10.0, 0.0], [0.0, 10.0], 0.9), [9.0, 1.0])
+
+
+# ----------------------------------------------------------------------------- backward pass
+
+def test_backward_against_finite_differences():
+    """The oracle's gradients against central differences of its own forward definition, in fp64
+    on a tiny layer (inputs chosen exactly representable in bf16 so that perturbations can be
+    applied to the widened values)."""
+    rng = np.random.default_rng(12)
+    T, K, E, d, f = 5, 2, 3, 4, 3
+    ids = np.array([rng.choice(E, size=K, replace=False) for _ in range(T)]).astype(np.int32)
+    gates = rng.random((T, K)).astype(np.float32)
+    xb = _bits(rng.standard_normal((T, d)))
+    w1b, w3b, w2b = _bits(rng.standard_normal((E, f, d))), _bits(rng.standard_normal((E, f, d))), _bits(rng.standard_normal((E, d, f)))
+    d_out = rng.standard_normal((T, d))
+    dx, dg, dw1, dw3, dw2 = O.moe_layer_backward(xb, ids, gates, w1b, w3b, w2b, d_out, E)
+
+    X, W1, W3, W2 = (W.bf16_bits_to_f64(a) for a in (xb, w1b, w3b, w2b))
+    G = gates.astype(np.float64)
+
+    def loss(X, G, W1, W3, W2):                                # scalar: <d_out, layer output>, plain fp64 definition
+        tot = 0.0
+        for t in range(T):
+            for k in range(K):
+                e = ids[t, k]
+                a, b = W1[e] @ X[t], W3[e] @ X[t]
+                tot += G[t, k] * float(d_out[t] @ (W2[e] @ (a / (1 + np.exp(-a)) * b)))
+        return tot
+
+    eps = 1e-6
+    def fd(arr, idx, pos):
+        args = [X.copy(), G.copy(), W1.copy(), W3.copy(), W2.copy()]
+        args[pos][idx] += eps
+        up = loss(*args)
+        args[pos][idx] -= 2 * eps
+        return (up - loss(*args)) / (2 * eps)
+
+    for arr, grad, pos in ((X, dx, 0), (G, dg, 1), (W1, dw1, 2), (W3, dw3, 3), (W2, dw2, 4)):
+        for idx in [tuple(rng.integers(0, n) for n in arr.shape) for _ in range(6)]:
+            assert grad[idx] == pytest.approx(fd(arr, idx, pos), rel=1e-5, abs=1e-7)
+    assert O.dsilu(np.array([0.0]))[0] == 0.5 and O.dsilu(np.array([40.0]))[0] == pytest.approx(1.0)
