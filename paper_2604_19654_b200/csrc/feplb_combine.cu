@@ -55,7 +55,7 @@ k_combine(const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_to_
       myg = 0.f;
       if (lane < K) {
         myrow = slot_to_row[(int64_t)t * K + lane];
-        myg = gates[(int64_t)t * K + lane];
+        myg = gates ? gates[(int64_t)t * K + lane] : 1.f;   // no gates: plain sum (backward of the dispatch)
       }
     }
     const bool on = c < chunks;

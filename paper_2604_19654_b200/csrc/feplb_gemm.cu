@@ -21,6 +21,7 @@
 #include <cstdio>
 
 #include "feplb_internal.h"
+#include "feplb_tc.cuh"
 
 namespace {
 
@@ -31,7 +32,6 @@ constexpr int kAccCols = 256;          // TMEM columns of one accumulator
 constexpr int kTmemCols = 512;         // all of TMEM: one CTA per SM
 constexpr int kABytes = BM * BK * 2;               // 16 KiB per sub-tile
 constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
-constexpr unsigned long long kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s per wait
 
 // Two forms of one kernel.
 //   single (PAIR = false): one CTA computes a 128 x 256 tile (UMMA M x N, cta_group::1); K step 64;
@@ -88,175 +88,9 @@ struct GemmParams {
   __nv_bfloat16* out;
   int ld_out;           // elements between output rows
   uint32_t* status;
+  __nv_bfloat16* ab_out;   // pass 1, optional: pre-activations a | b saved for the backward pass ([rows, 2f])
 };
 
-// ------------------------------------------------------------------------------------------ PTX
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting or the limit expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status,
-                                          unsigned long long limit_ns = kWaitLimitNs) {
-  if (mbar_try_wait(bar, parity)) return true;
-  unsigned long long t0 = 0;
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > limit_ns) {
-        *abort_flag = 1;
-        atomicOr(status, FEPLB_ST_WAIT);
-        return false;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
-  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
-}
-
-// 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier of this CTA.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate, issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The mbarrier receives one arrival once all tcgen05.mma issued so far by this thread are done.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns of TMEM -> 32 registers per thread (thread i = lane i).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// ---- cluster-of-two forms (cta_group::2) --------------------------------------------------------
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// TMA load into this CTA's shared memory whose byte count is credited to an mbarrier that may
-// live in the peer CTA of the pair (cluster address).
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-// D[tmem of both CTAs] (+)= A[256 rows, 128 per CTA] * B[N columns, N/2 per CTA]
-__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// One arrival on the mbarrier at this offset in BOTH CTAs of the pair once the MMAs issued so far are done.
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"((unsigned short)3) : "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) wide and
-// 128-byte swizzled, 8-row groups 1024 bytes apart: start address >> 4 in bits [0,14), leading
-// byte offset (unused for swizzled K-major) = 1 in [16,30), stride byte offset 1024 >> 4 in
-// [32,46), descriptor version 1 in [46,48), layout type 2 (SWIZZLE_128B) in [61,64).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-// Instruction descriptor of tcgen05.mma kind::f16: D fp32 (bits [4,6) = 1), A and B bf16
-// ([7,10) = 1, [10,13) = 1), both K-major (bits 15, 16 = 0), N >> 3 in [17,23), M >> 4 in [24,29).
-__device__ __forceinline__ uint32_t make_idesc(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
-__device__ __forceinline__ float silu_f(float a) { return __fdividef(a, 1.f + __expf(-a)); }
 
 struct TileCoord { int row0, rows_valid, expert, slot, nt; };   // slot >= 0: weights in that receive slot
 
@@ -292,6 +126,30 @@ __device__ __forceinline__ void convert_slice(const uint32_t (&a)[32], const uin
     }
     packed[i] = pack_bf16x2(v0, v1);
   }
+}
+
+// 32 rows x 64 bf16 columns, one row per lane in packed[32]: through the warp's staging area (row
+// `lane`, 16-byte chunk j at position j ^ (lane & 7)) and out again 4 rows per instruction, so
+// that every global store covers whole 128-byte lines; rows >= rows_here are not written.
+__device__ __forceinline__ void stage_and_store(uint32_t stg, const uint32_t* packed, __nv_bfloat16* obase, int ld,
+                                                int col, int rows_here, int lane) {
+  const int rd_row = lane >> 3, rd_chunk = lane & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(packed[4 * j]), "r"(packed[4 * j + 1]),
+                 "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
+  }
+  __syncwarp();
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int r = it * 4 + rd_row;
+    const uint32_t addr = stg + (uint32_t)(r * 128 + ((rd_chunk ^ (r & 7)) << 4));
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    if (r < rows_here) *reinterpret_cast<uint4*>(obase + (int64_t)r * ld + col + rd_chunk * 8) = v;
+  }
+  __syncwarp();
 }
 
 template <bool SWIGLU, bool PAIR>
@@ -478,7 +336,6 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int q = warp & 3;                   // TMEM lane quarter this warp may read
     const uint32_t stg = smem_u32(epi_smem + (size_t)(warp - 2) * kEpiStageBytes);
     const int out_cols = SWIGLU ? p.bn : 2 * p.bn;
-    const int rd_row = lane >> 3, rd_chunk = lane & 7;   // read-back role: 4 rows x 8 chunks per step
     int as = 0;
     uint32_t aphase = 0;
     bool ok = true;
@@ -501,6 +358,24 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       for (int col = 0; col < out_cols; col += 64) {
         tmem_ld_wait();
+        if (SWIGLU && p.ab_out != nullptr) {
+          // training: also keep the pre-activations a | b of these 64 hidden units (bf16) for the
+          // backward pass, in [rows, 2f] with b at column offset f
+          __nv_bfloat16* abase = p.ab_out + (int64_t)(c.row0 + row_off) * (2 * p.ld_out);
+          const int hcol = c.nt * out_cols + col;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            packed[i] = pack_bf16x2(__uint_as_float(a0[2 * i]), __uint_as_float(a0[2 * i + 1]));
+            packed[16 + i] = pack_bf16x2(__uint_as_float(a1[2 * i]), __uint_as_float(a1[2 * i + 1]));
+          }
+          stage_and_store(stg, packed, abase, 2 * p.ld_out, hcol, rows_here, lane);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            packed[i] = pack_bf16x2(__uint_as_float(b0[2 * i]), __uint_as_float(b0[2 * i + 1]));
+            packed[16 + i] = pack_bf16x2(__uint_as_float(b1[2 * i]), __uint_as_float(b1[2 * i + 1]));
+          }
+          stage_and_store(stg, packed, abase, 2 * p.ld_out, p.ld_out + hcol, rows_here, lane);
+        }
         convert_slice<SWIGLU>(a0, b0, packed);
         convert_slice<SWIGLU>(a1, b1, packed + 16);
         if (col + 64 < out_cols) {           // next slice's TMEM loads fly while this one is stored
@@ -511,24 +386,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             tmem_ld32(taddr + (uint32_t)(p.bn + col + 96), b1);
           }
         }
-        // row `lane`: chunk j (columns 8j..8j+7) goes to position j ^ (lane & 7)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(packed[4 * j]), "r"(packed[4 * j + 1]),
-                       "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
-        }
-        __syncwarp();
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int r = it * 4 + rd_row;
-          const uint32_t addr = stg + (uint32_t)(r * 128 + ((rd_chunk ^ (r & 7)) << 4));
-          uint4 v;
-          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-          if (r < rows_here)
-            *reinterpret_cast<uint4*>(obase + (int64_t)r * p.ld_out + col + rd_chunk * 8) = v;
-        }
-        __syncwarp();
+        stage_and_store(stg, packed, obase, p.ld_out, col, rows_here, lane);
       }
       tc_fence_before();
       __syncwarp();
@@ -667,10 +525,10 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p1.n_recv_slots = has_recv ? a.n_recv_slots : 0;
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
   p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1;
-  p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status;
+  p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status; p1.ab_out = (__nv_bfloat16*)a.ab_out;
   GemmParams p2 = p1;
   p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
-  p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d;
+  p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d; p2.ab_out = nullptr;
 
   cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st)
                          : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st);

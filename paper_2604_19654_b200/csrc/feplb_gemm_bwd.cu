@@ -1,0 +1,617 @@
+// Backward pass of the grouped SwiGLU expert FFN on sm_100a (the paper reports backward layer times
+// in Table 2 but does not describe the pass; this is the derivative of the forward definition,
+// computed over the same groups).  One warp-specialised tcgen05 kernel in three kinds, all with
+// K-major operands staged by TMA (weights and activations are transposed beforehand where the
+// contraction runs over their slow dimension):
+//   DH: dH = dY W2 (A = dY rows, B = W2^T tiles), epilogue applies the SwiGLU derivative with the
+//       saved pre-activations:  dA = dH * b * silu'(a),  dB = dH * silu(a)  -> dAB [rows, 2f]
+//   DX: dX = dA W1^T + dB W3^T as ONE contraction over K = 2f ([dA|dB] against W1^T then W3^T)
+//   WG: weight gradients, one (expert, M tile, N tile) per tile with the contraction running over
+//       that expert's rows:  dW[e] = P_e^T Q_e  (fp32 out, optionally accumulated), operands are
+//       the transposed activations P^T [M, rows], Q^T [N, rows]
+// Pipeline as in the forward kernel: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps
+// 2..5 epilogue; 4-stage ring of 48 KiB; two TMEM accumulators; every mbarrier wait bounded.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+
+#include "feplb_internal.h"
+#include "feplb_tc.cuh"
+
+namespace {
+
+enum { KIND_DH = 0, KIND_DX = 1, KIND_WG = 2 };
+
+constexpr int BM = FEPLB_TILE_M;
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
+constexpr int kAccCols = 256;
+constexpr int kTmemCols = 512;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kBBytesMax = 256 * BK * 2;
+constexpr int kStages = 4;
+constexpr int kAccStages = 2;
+constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kEpiStageBytes = 32 * 128;
+
+struct Tail {
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long tmem_full[kAccStages];
+  unsigned long long tmem_empty[kAccStages];
+  uint32_t tmem_base;
+  int abort_flag;
+  int prefix[FEPLB_MAX_GROUPS + 1];
+  int g_row_start[FEPLB_MAX_GROUPS];
+  int g_rows[FEPLB_MAX_GROUPS];
+  int g_expert[FEPLB_MAX_GROUPS];
+};
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (size_t)kEpiWarps * kEpiStageBytes + sizeof(Tail);
+static_assert(kSmemBytes <= 232448 && kSmemBytes > 116 * 1024, "one CTA per SM: each allocates all of TMEM");
+
+struct BwdParams {
+  const feplb_group* groups;   // DH/DX: the group table; WG: the E-entry home table (one entry per expert)
+  int n_groups;
+  int which;
+  int E;
+  int64_t s_cap;
+  int n_tiles_n;               // N tiles per M tile
+  int num_k_blocks;            // DH: d/64, DX: 2f/64, WG: unused (ceil(rows/64) per expert)
+  int k_switch;                // DX: first K block served by the second B map (f/64)
+  int n_limit;                 // DH/DX: valid output columns (a last N tile may overhang)
+  int b_rows_per_expert;       // DH: f, DX: d, WG: 0 (B^T is not per expert)
+  int bn;                      // rows of one B half tile; the MMA has N = 2*bn
+  __nv_bfloat16* out;          // DH: dAB [s_cap, 2f]; DX: dX_perm [s_cap, d]
+  int ld_out;
+  const __nv_bfloat16* ab;     // DH: saved pre-activations [s_cap, 2f] (a | b)
+  int f;                       // DH: columns of a (and offset of b)
+  float* wout;                 // WG: fp32 [E, m_total, n_total]
+  int m_total, n_total;        // WG
+  int m_tiles;                 // WG: M tiles per expert
+  int accumulate;              // WG: add to wout instead of overwriting it
+  uint32_t* status;
+};
+
+struct Coord { int row0, rows_valid, expert, mt, nt, kblocks; };
+
+template <int KIND>
+__device__ __forceinline__ Coord tile_coord(const Tail* t, const BwdParams& p, int tile) {
+  Coord c;
+  if (KIND == KIND_WG) {
+    const int per = p.m_tiles * p.n_tiles_n;
+    const int g = tile / per;
+    const int r = tile - g * per;
+    c.mt = r / p.n_tiles_n;
+    c.nt = r - c.mt * p.n_tiles_n;
+    c.expert = t->g_expert[g];
+    c.row0 = t->g_row_start[g];               // first row of the expert's segment = start of its K range
+    c.rows_valid = t->g_rows[g];
+    c.kblocks = (t->g_rows[g] + BK - 1) / BK;
+    return c;
+  }
+  const int mt = tile / p.n_tiles_n;
+  int lo = 0, hi = p.n_groups;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (t->prefix[mid] <= mt) lo = mid; else hi = mid;
+  }
+  const int local = mt - t->prefix[lo];
+  c.row0 = t->g_row_start[lo] + local * BM;
+  c.rows_valid = min(BM, t->g_rows[lo] - local * BM);
+  c.expert = t->g_expert[lo];
+  c.mt = mt;
+  c.nt = tile - mt * p.n_tiles_n;
+  c.kblocks = p.num_k_blocks;
+  return c;
+}
+
+__device__ __forceinline__ float sigmoid_f(float a) { return __fdividef(1.f, 1.f + __expf(-a)); }
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// Stage 32 rows x 64 bf16 columns (packed[32] per lane = its row) through the warp's swizzled
+// staging area and write them out 4 rows per instruction, whole 128-byte lines, row-masked.
+__device__ __forceinline__ void staged_store(uint32_t stg, const uint32_t* packed, __nv_bfloat16* obase, int ld_out,
+                                             int col, int rows_here, int lane) {
+  const int rd_row = lane >> 3, rd_chunk = lane & 7;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(packed[4 * j]), "r"(packed[4 * j + 1]),
+                 "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
+  }
+  __syncwarp();
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int r = it * 4 + rd_row;
+    const uint32_t addr = stg + (uint32_t)(r * 128 + ((rd_chunk ^ (r & 7)) << 4));
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    if (r < rows_here) *reinterpret_cast<uint4*>(obase + (int64_t)r * ld_out + col + rd_chunk * 8) = v;
+  }
+  __syncwarp();
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+               const __grid_constant__ CUtensorMap tm_b1, const BwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* epi_smem = smem + (size_t)kStages * kStageBytes;
+  Tail* tail = reinterpret_cast<Tail*>(epi_smem + (size_t)kEpiWarps * kEpiStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &tail->abort_flag;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_b0);
+    prefetch_tmap(&tm_b1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&tail->full[s]), 1);
+      mbar_init(smem_u32(&tail->empty[s]), 1);
+    }
+    for (int a = 0; a < kAccStages; ++a) {
+      mbar_init(smem_u32(&tail->tmem_full[a]), 1);
+      mbar_init(smem_u32(&tail->tmem_empty[a]), kEpiWarps);
+    }
+    tail->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  for (int g = threadIdx.x; g < p.n_groups; g += kThreads) {
+    const feplb_group gr = p.groups[g];
+    const bool selected = p.which == FEPLB_FFN_ALL || (p.which == FEPLB_FFN_STATIC) == (gr.is_dynamic == 0);
+    int tiles = 0, rows = 0;
+    if (selected && gr.rows > 0) {
+      const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 && (int64_t)gr.row_start + gr.rows <= p.s_cap;
+      if (ok) { tiles = (gr.rows + BM - 1) / BM; rows = gr.rows; }
+      else atomicOr(p.status, FEPLB_ST_GROUP);
+    }
+    tail->prefix[g + 1] = tiles;
+    tail->g_row_start[g] = gr.row_start;
+    tail->g_rows[g] = rows;                      // 0 for unselected or malformed entries
+    tail->g_expert[g] = gr.expert;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    const int per = (p.n_groups + 31) / 32;
+    const int g0 = lane * per, g1 = min(p.n_groups, g0 + per);
+    int sum = 0;
+    for (int g = g0; g < g1; ++g) sum += tail->prefix[g + 1];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    int run = incl - sum;
+    for (int g = g0; g < g1; ++g) {
+      const int t = tail->prefix[g + 1];
+      run += t;
+      tail->prefix[g + 1] = run;
+    }
+    if (lane == 0) tail->prefix[0] = 0;
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  const int total_tiles = KIND == KIND_WG ? p.n_groups * p.m_tiles * p.n_tiles_n : tail->prefix[p.n_groups] * p.n_tiles_n;
+  const uint32_t b_half_bytes = (uint32_t)p.bn * BK * 2;
+  const uint32_t stage_tx = kABytes + 2 * b_half_bytes;
+
+  if (warp == 0) {
+    // ---- TMA producer ---------------------------------------------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const Coord c = tile_coord<KIND>(tail, p, tile);
+        for (int kb = 0; kb < c.kblocks; ++kb) {
+          if (!(ok = mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status))) break;
+          const uint32_t full = smem_u32(&tail->full[stage]);
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
+          const uint32_t sb = sa + kABytes;
+          mbar_expect_tx(full, stage_tx);
+          if (KIND == KIND_WG) {
+            // K runs along the expert's rows (inner dimension of the transposed activations)
+            const int k0 = c.row0 + kb * BK;
+            tma_load_2d(sa, &tm_a, full, k0, c.mt * BM);
+            tma_load_2d(sb, &tm_b0, full, k0, c.nt * 2 * p.bn);
+            tma_load_2d(sb + b_half_bytes, &tm_b0, full, k0, c.nt * 2 * p.bn + p.bn);
+          } else {
+            const CUtensorMap* mb = (KIND == KIND_DX && kb >= p.k_switch) ? &tm_b1 : &tm_b0;
+            const int kb_b = (KIND == KIND_DX && kb >= p.k_switch) ? kb - p.k_switch : kb;
+            const int brow = c.expert * p.b_rows_per_expert + c.nt * 2 * p.bn;
+            tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
+            tma_load_2d(sb, mb, full, kb_b * BK, brow);
+            tma_load_2d(sb + b_half_bytes, mb, full, kb_b * BK, brow + p.bn);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(100);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer -------------------------------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(BM, 2 * p.bn);
+      int stage = 0, as = 0;
+      uint32_t phase = 0, aphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const Coord c = tile_coord<KIND>(tail, p, tile);
+        if (!(ok = mbar_wait(smem_u32(&tail->tmem_empty[as]), aphase ^ 1u, abort_flag, p.status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(as * kAccCols);
+        for (int kb = 0; kb < c.kblocks; ++kb) {
+          if (!(ok = mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+          umma_commit(smem_u32(&tail->empty[stage]));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (c.kblocks > 0) umma_commit(smem_u32(&tail->tmem_full[as]));
+        else mbar_arrive(smem_u32(&tail->tmem_full[as]));     // an expert without rows: nothing was issued
+        if (++as == kAccStages) { as = 0; aphase ^= 1u; }
+      }
+    }
+  } else {
+    // ---- epilogue -----------------------------------------------------------------------------
+    const int q = warp & 3;
+    const uint32_t stg = smem_u32(epi_smem + (size_t)(warp - 2) * kEpiStageBytes);
+    int as = 0;
+    uint32_t aphase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      const Coord c = tile_coord<KIND>(tail, p, tile);
+      ok = mbar_wait(smem_u32(&tail->tmem_full[as]), aphase, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * kAccCols);
+      const int out_cols = 2 * p.bn;
+      if (KIND == KIND_WG) {
+        // fp32 tile of dW[e]: thread = row of the M tile, 32 consecutive columns = one 128-byte line
+        const int m = c.mt * BM + q * 32 + lane;
+        float* orow = p.wout + ((int64_t)c.expert * p.m_total + m) * p.n_total + (int64_t)c.nt * out_cols;
+        for (int col = 0; col < out_cols; col += 32) {
+          uint32_t a[32];
+          if (c.kblocks > 0) {
+            tmem_ld32(taddr + (uint32_t)col, a);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) a[i] = 0u;
+          }
+          const int n0 = c.nt * out_cols + col;
+          if (m < p.m_total && n0 < p.n_total) {      // n_total is a multiple of 32
+            float4* dst = reinterpret_cast<float4*>(orow + col);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float4 v = make_float4(__uint_as_float(a[4 * i]), __uint_as_float(a[4 * i + 1]),
+                                     __uint_as_float(a[4 * i + 2]), __uint_as_float(a[4 * i + 3]));
+              if (p.accumulate) {
+                const float4 o = dst[i];
+                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+              }
+              dst[i] = v;
+            }
+          }
+        }
+      } else {
+        const int row_off = q * 32;
+        const int rows_here = c.rows_valid - row_off;
+        const int my_row = c.row0 + row_off + lane;
+        const bool row_ok = lane < rows_here;
+        for (int col = 0; col < out_cols; col += 64) {
+          uint32_t a0[32], a1[32];
+          tmem_ld32(taddr + (uint32_t)col, a0);
+          tmem_ld32(taddr + (uint32_t)(col + 32), a1);
+          tmem_ld_wait();
+          const int gcol = c.nt * out_cols + col;      // first of this slice's 64 output columns
+          if (gcol >= p.n_limit) continue;             // overhang of the last N tile (warp-uniform)
+          if (KIND == KIND_DX) {
+            uint32_t packed[32];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              packed[i] = pack_bf16x2(__uint_as_float(a0[2 * i]), __uint_as_float(a0[2 * i + 1]));
+              packed[16 + i] = pack_bf16x2(__uint_as_float(a1[2 * i]), __uint_as_float(a1[2 * i + 1]));
+            }
+            staged_store(stg, packed, p.out + (int64_t)(c.row0 + row_off) * p.ld_out, p.ld_out, gcol, rows_here, lane);
+          } else {
+            // SwiGLU derivative: this thread's row, 64 columns of a and b (128 bytes each)
+            uint32_t pa[32], pb[32];
+            if (row_ok) {
+              const uint4* ap = reinterpret_cast<const uint4*>(p.ab + (int64_t)my_row * (2 * p.f) + gcol);
+              const uint4* bp = reinterpret_cast<const uint4*>(p.ab + (int64_t)my_row * (2 * p.f) + p.f + gcol);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const uint4 va = ap[i], vb = bp[i];
+                pa[4 * i] = va.x; pa[4 * i + 1] = va.y; pa[4 * i + 2] = va.z; pa[4 * i + 3] = va.w;
+                pb[4 * i] = vb.x; pb[4 * i + 1] = vb.y; pb[4 * i + 2] = vb.z; pb[4 * i + 3] = vb.w;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) { pa[i] = 0u; pb[i] = 0u; }
+            }
+            uint32_t pda[32], pdb[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float dh0 = __uint_as_float(i < 16 ? a0[2 * i] : a1[2 * (i - 16)]);
+              const float dh1 = __uint_as_float(i < 16 ? a0[2 * i + 1] : a1[2 * (i - 16) + 1]);
+              const float x0 = bf16_lo(pa[i]), x1 = bf16_hi(pa[i]);
+              const float y0 = bf16_lo(pb[i]), y1 = bf16_hi(pb[i]);
+              const float s0 = sigmoid_f(x0), s1 = sigmoid_f(x1);
+              // silu(a) = a*s;  silu'(a) = s * (1 + a * (1 - s))
+              pda[i] = pack_bf16x2(dh0 * y0 * s0 * (1.f + x0 * (1.f - s0)), dh1 * y1 * s1 * (1.f + x1 * (1.f - s1)));
+              pdb[i] = pack_bf16x2(dh0 * x0 * s0, dh1 * x1 * s1);
+            }
+            __nv_bfloat16* obase = p.out + (int64_t)(c.row0 + row_off) * p.ld_out;
+            staged_store(stg, pda, obase, p.ld_out, gcol, rows_here, lane);
+            staged_store(stg, pdb, obase, p.ld_out, p.f + gcol, rows_here, lane);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      if (++as == kAccStages) { as = 0; aphase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- bandwidth kernels of the backward pass ---------------------------------------------------
+
+// dst[c, r] = src[r, c] for a batch of bf16 matrices (32 x 32 tiles through shared memory).  With
+// row_token != nullptr, source rows that hold no token (row_token[r] < 0: the padding at the end
+// of an expert's segment, never written by the masked stores of the GEMMs) are transposed as
+// zeros, so that they add nothing to a contraction over rows.
+__global__ void __launch_bounds__(256)
+k_transpose_bf16(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows, int cols,
+                 int64_t ld_src, int64_t ld_dst, int64_t batch_src, int64_t batch_dst,
+                 const int32_t* __restrict__ row_token) {
+  __shared__ __nv_bfloat16 t[32][34];
+  src += (int64_t)blockIdx.z * batch_src;
+  dst += (int64_t)blockIdx.z * batch_dst;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;    // 32 x 8
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + ty + 8 * i, c = c0 + tx;
+    const bool live = r < rows && c < cols && (row_token == nullptr || row_token[r] >= 0);
+    t[ty + 8 * i][tx] = live ? src[(int64_t)r * ld_src + c] : __float2bfloat16(0.f);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = c0 + ty + 8 * i, r = r0 + tx;
+    if (c < cols && r < rows) dst[(int64_t)c * ld_dst + r] = t[tx][ty + 8 * i];
+  }
+}
+
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// Backward of the combine: for every slot (t, k) with row r = slot_to_row[t, k]
+//   dY_perm[r, :] = gates[t, k] * dOut[t, :]         dGates[t, k] = <dOut[t, :], y_perm[r, :]>
+// One warp per slot, slots dealt out in equal contiguous ranges.
+__global__ void __launch_bounds__(256)
+k_combine_bwd(const uint4* __restrict__ d_out, const uint4* __restrict__ y_perm, const int32_t* __restrict__ slot_to_row,
+              const float* __restrict__ gates, uint4* __restrict__ d_y_perm, float* __restrict__ d_gates,
+              int64_t S, int K, int chunks) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * 256) >> 5;
+  const int64_t s0 = S * warp / nwarps, s1 = S * (warp + 1) / nwarps;
+  for (int64_t s = s0; s < s1; ++s) {
+    const int row = slot_to_row[s];
+    const float g = gates[s];
+    const int64_t t = s / K;
+    float dot = 0.f;
+    if (row >= 0) {
+      for (int c = lane; c < chunks; c += 32) {
+        const uint4 o = ld_nc_v4(d_out + t * chunks + c);
+        const uint4 y = ld_nc_v4(y_perm + (int64_t)row * chunks + c);
+        uint4 w;
+        const uint32_t ov[4] = {o.x, o.y, o.z, o.w}, yv[4] = {y.x, y.y, y.z, y.w};
+        uint32_t wv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float o0 = bf16_lo(ov[i]), o1 = bf16_hi(ov[i]);
+          dot = fmaf(o0, bf16_lo(yv[i]), dot);
+          dot = fmaf(o1, bf16_hi(yv[i]), dot);
+          wv[i] = pack_bf16x2(g * o0, g * o1);
+        }
+        w.x = wv[0]; w.y = wv[1]; w.z = wv[2]; w.w = wv[3];
+        d_y_perm[(int64_t)row * chunks + c] = w;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (lane == 0) d_gates[s] = row >= 0 ? dot : 0.f;
+  }
+}
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_fn() {
+  static encode_tiled_fn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_tiled_fn>(p);
+  }
+  return fn;
+}
+
+// Row-major bf16 matrix [rows, inner] with a row pitch of ld elements -> [box_rows, 64] boxes, 128-byte swizzle.
+bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, uint64_t ld, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KIND>
+cudaError_t launch_kind(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const BwdParams& p,
+                        int grid, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_ffn_bwd_gemm<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  k_ffn_bwd_gemm<KIND><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, p);
+  return cudaGetLastError();
+}
+
+cudaError_t transpose(const void* src, void* dst, int rows, int cols, int64_t ld_src, int64_t ld_dst, int batch,
+                      int64_t batch_src, int64_t batch_dst, cudaStream_t st, int64_t* n_launch,
+                      const int32_t* row_token = nullptr) {
+  if (rows == 0 || cols == 0 || batch == 0) return cudaSuccess;
+  dim3 grid((cols + 31) / 32, (rows + 31) / 32, batch);
+  k_transpose_bf16<<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, cols, ld_src, ld_dst,
+                                         batch_src, batch_dst, row_token);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t feplb_launch_transpose_weights(const void* w1, const void* w3, const void* w2, void* w1t, void* w3t, void* w2t,
+                                           int E, int d, int f, cudaStream_t st, int64_t* n_launch) {
+  const int64_t per = (int64_t)d * f;
+  cudaError_t e = transpose(w1, w1t, f, d, d, f, E, per, per, st, n_launch);       // [E,f,d] -> [E,d,f]
+  if (e == cudaSuccess) e = transpose(w3, w3t, f, d, d, f, E, per, per, st, n_launch);
+  if (e == cudaSuccess) e = transpose(w2, w2t, d, f, f, d, E, per, per, st, n_launch);   // [E,d,f] -> [E,f,d]
+  return e;
+}
+
+cudaError_t feplb_launch_combine_bwd(const void* d_out, const void* y_perm, const int32_t* slot_to_row, const float* gates,
+                                     void* d_y_perm, float* d_gates, int T, int K, int d, int num_sms, cudaStream_t st,
+                                     int64_t* n_launch) {
+  const int64_t S = (int64_t)T * K;
+  if (S == 0) return cudaSuccess;
+  int blocks = num_sms * 6;
+  const int64_t need = (S + 7) / 8;
+  if (need < blocks) blocks = (int)need;
+  k_combine_bwd<<<blocks, 256, 0, st>>>((const uint4*)d_out, (const uint4*)y_perm, slot_to_row, gates, (uint4*)d_y_perm,
+                                        d_gates, S, K, d / 8);
+  ++*n_launch;
+  return cudaGetLastError();
+}
+
+int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn) {
+  if (a.n_groups == 0 || a.s_cap == 0) return FEPLB_OK;
+  const int d = a.d, f = a.f;
+  cudaError_t e = cudaSuccess;
+  auto fail_cuda = [&](const char* what) {
+    snprintf(err, errn, "%s: %s", what, cudaGetErrorString(e));
+    return FEPLB_E_CUDA;
+  };
+  // ---- dH and the SwiGLU derivative: dAB = SwiGLU'(a, b; dY W2) ----------------------------------
+  const int bn_h = (f % 256 == 0) ? 128 : 64;      // N = f in tiles of 2*bn columns (the last may overhang)
+  const int bn_x = (d % 256 == 0) ? 128 : 64;
+  CUtensorMap tm_dy, tm_w2t, tm_dab, tm_w1t, tm_w3t;
+  if (!make_tmap(&tm_dy, a.d_y_perm, (uint64_t)a.s_cap, (uint64_t)d, (uint64_t)d, BM) ||
+      !make_tmap(&tm_w2t, a.w2t, (uint64_t)a.E * f, (uint64_t)d, (uint64_t)d, bn_h) ||
+      !make_tmap(&tm_dab, a.d_ab, (uint64_t)a.s_cap, (uint64_t)2 * f, (uint64_t)2 * f, BM) ||
+      !make_tmap(&tm_w1t, a.w1t, (uint64_t)a.E * d, (uint64_t)f, (uint64_t)f, bn_x) ||
+      !make_tmap(&tm_w3t, a.w3t, (uint64_t)a.E * d, (uint64_t)f, (uint64_t)f, bn_x)) {
+    snprintf(err, errn, "cuTensorMapEncodeTiled failed (backward)");
+    return FEPLB_E_CUDA;
+  }
+  BwdParams p = {};
+  p.groups = a.groups; p.n_groups = a.n_groups; p.which = a.which; p.E = a.E; p.s_cap = a.s_cap; p.status = a.status;
+  BwdParams ph = p;
+  ph.n_tiles_n = (f + 2 * bn_h - 1) / (2 * bn_h); ph.n_limit = f; ph.num_k_blocks = d / BK; ph.b_rows_per_expert = f; ph.bn = bn_h;
+  ph.out = (__nv_bfloat16*)a.d_ab; ph.ld_out = 2 * f; ph.ab = (const __nv_bfloat16*)a.ab_saved; ph.f = f;
+  e = launch_kind<KIND_DH>(tm_dy, tm_w2t, tm_w2t, ph, a.num_sms, st);
+  ++*n_launch;
+  if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DH>");
+  // ---- dX = [dA | dB] [W1^T ; W3^T] ------------------------------------------------------------------
+  BwdParams px = p;
+  px.n_tiles_n = d / (2 * bn_x); px.n_limit = d; px.num_k_blocks = 2 * f / BK; px.k_switch = f / BK; px.b_rows_per_expert = d; px.bn = bn_x;
+  px.out = (__nv_bfloat16*)a.d_x_perm; px.ld_out = d;
+  e = launch_kind<KIND_DX>(tm_dab, tm_w1t, tm_w3t, px, a.num_sms, st);
+  ++*n_launch;
+  if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DX>");
+  if (!a.dw1) return FEPLB_OK;
+  // ---- weight gradients: contraction over each expert's rows, on transposed activations -----------------
+  const int64_t ld_t = a.ld_t;     // row pitch of the transposed scratch (>= s_cap, multiple of 64)
+  char* tbuf = (char*)a.t_scratch;
+  void* xt = tbuf;                                                   // [d, ld_t]
+  void* ht = tbuf + (size_t)d * ld_t * 2;                            // [f, ld_t]
+  void* dyt = tbuf + (size_t)(d + f) * ld_t * 2;                     // [d, ld_t]
+  void* dabt = tbuf + (size_t)(2 * d + f) * ld_t * 2;                // [2f, ld_t]
+  const int rows = (int)a.s_cap;
+  e = transpose(a.x_perm, xt, rows, d, d, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
+  if (e == cudaSuccess) e = transpose(a.h, ht, rows, f, f, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
+  if (e == cudaSuccess) e = transpose(a.d_y_perm, dyt, rows, d, d, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
+  if (e == cudaSuccess) e = transpose(a.d_ab, dabt, rows, 2 * f, 2 * f, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
+  if (e != cudaSuccess) return fail_cuda("k_transpose_bf16");
+  // dW2[e] [d, f] = dY_e^T H_e;   dW1[e] [f, d] = dA_e^T X_e;   dW3[e] [f, d] = dB_e^T X_e
+  struct WG { const void* at; int m_total; const void* bt; int n_total; float* out; };
+  const WG jobs[3] = {
+      {dyt, d, ht, f, a.dw2},
+      {dabt, f, xt, d, a.dw1},
+      {(const char*)dabt + (size_t)f * ld_t * 2, f, xt, d, a.dw3},
+  };
+  for (const WG& j : jobs) {
+    const int bn = (j.n_total % 256 == 0) ? 128 : 64;
+    CUtensorMap tm_at, tm_bt;
+    if (!make_tmap(&tm_at, j.at, (uint64_t)j.m_total, (uint64_t)a.s_cap, (uint64_t)ld_t, BM) ||
+        !make_tmap(&tm_bt, j.bt, (uint64_t)j.n_total, (uint64_t)a.s_cap, (uint64_t)ld_t, bn)) {
+      snprintf(err, errn, "cuTensorMapEncodeTiled failed (weight gradient)");
+      return FEPLB_E_CUDA;
+    }
+    BwdParams pw = p;
+    pw.groups = a.expert_table; pw.n_groups = a.E; pw.which = FEPLB_FFN_ALL;
+    pw.bn = bn; pw.n_tiles_n = (j.n_total + 2 * bn - 1) / (2 * bn); pw.m_tiles = (j.m_total + BM - 1) / BM;
+    pw.m_total = j.m_total; pw.n_total = j.n_total; pw.wout = j.out; pw.accumulate = a.accumulate;
+    e = launch_kind<KIND_WG>(tm_at, tm_bt, tm_bt, pw, a.num_sms, st);
+    ++*n_launch;
+    if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<WG>");
+  }
+  return FEPLB_OK;
+}

@@ -68,11 +68,31 @@ struct feplb_gemm_args {
   int pair;   // 1: clusters of two CTAs on 256-row tiles (cta_group::2); 0: one CTA per 128-row tile
   // receive buffer of migrated experts' weights ([n_recv_slots, f, d] x2 and [n_recv_slots, d, f]); may be null
   const void* recv_w1; const void* recv_w3; const void* recv_w2; int n_recv_slots;
+  void* ab_out;   // optional [s_cap, 2f]: pass 1 also saves the pre-activations a | b (for the backward pass)
 };
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
 // One thread waits (bounded by limit_ns) on an mbarrier nobody completes; *gave_up = 1 and FEPLB_ST_WAIT expected.
 cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up, cudaStream_t st);
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
+// ---- backward pass ---------------------------------------------------------------------------
+struct feplb_bwd_args {
+  const void* x_perm; const void* ab_saved; const void* h; const void* d_y_perm;
+  const void* w1t; const void* w3t; const void* w2t;        // [E,d,f], [E,d,f], [E,f,d]
+  const feplb_group* groups; int n_groups; int which;
+  const feplb_group* expert_table;                          // E entries {e, first row, rows}: the K ranges of the weight gradients
+  const int32_t* row_to_token;
+  void* d_ab; void* d_x_perm;                               // [s_cap, 2f], [s_cap, d]
+  float* dw1; float* dw3; float* dw2; int accumulate;       // fp32 [E,f,d], [E,f,d], [E,d,f]; dw1 == nullptr: skip
+  void* t_scratch; int64_t ld_t;                            // transposed activations: (2d + 3f) rows of ld_t bf16
+  int E, d, f; int64_t s_cap;
+  uint32_t* status; int num_sms;
+};
+cudaError_t feplb_launch_transpose_weights(const void* w1, const void* w3, const void* w2, void* w1t, void* w3t, void* w2t,
+                                           int E, int d, int f, cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_combine_bwd(const void* d_out, const void* y_perm, const int32_t* slot_to_row, const float* gates,
+                                     void* d_y_perm, float* d_gates, int T, int K, int d, int num_sms, cudaStream_t st,
+                                     int64_t* n_launch);
+int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
 #endif
 
 #endif  // FEPLB_INTERNAL_H_
