@@ -267,6 +267,9 @@ def run_cuda(args, w):
     strag = None
     if rank == 0 and not args.no_straggler and not args.quick:
         strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb)
+    args.backward_result = None
+    if rank == 0 and args.backward:
+        args.backward_result = measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, min(args.steps, 100))
     _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals, n_fw, e2e_value, h2d, d2h, strag, weights, n_mb)
     ctx.close()
     if world > 1:
@@ -326,6 +329,55 @@ def run_sweep(args):
         ctx.close()
         del buf, dev
         torch.cuda.empty_cache()
+
+
+def measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, steps):
+    """Forward + backward of the layer (weight gradients included, so expert segments are padded
+    to 128 rows), timed per phase with CUDA events on the launching stream."""
+    import torch
+    cfg = F.config_from_workload(w, row_align=128)
+    ctx, buf, bwd = F.Context(cfg), F.Buffers(cfg), F.BackwardBuffers(cfg)
+    ctx.set_preact_buffer(bwd.ab)
+    w1t = torch.empty(w.E, w.d, w.f, dtype=torch.bfloat16, device="cuda")
+    w3t = torch.empty_like(w1t)
+    w2t = torch.empty(w.E, w.f, w.d, dtype=torch.bfloat16, device="cuda")
+    ctx.transpose_weights(d_w1, d_w3, d_w2, w1t, w3t, w2t, stream=stream)
+    dw1 = torch.zeros(w.E, w.f, w.d, dtype=torch.float32, device="cuda")
+    dw3 = torch.zeros_like(dw1)
+    dw2 = torch.zeros(w.E, w.d, w.f, dtype=torch.float32, device="cuda")
+    d_out = [torch.randn(w.T, w.d, device="cuda", dtype=torch.float32).mul_(0.02).to(torch.bfloat16) for _ in range(2)]
+
+    def fwd(i):
+        x, ids, g = dev[i % n_mb]
+        ctx.moe_forward(x, ids, g, d_w1, d_w3, d_w2, buf, want_plan=False, stream=stream)
+
+    def back(i):
+        ctx.moe_backward(d_out[i & 1], dev[i % n_mb][2], w1t, w3t, w2t, buf, bwd, dw1, dw3, dw2, accumulate=True, stream=stream)
+
+    for i in range(3):
+        fwd(i)
+        back(i)
+    ctx.check_status()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    torch.cuda.synchronize()
+    for i in range(steps):
+        ev[i][0].record(stream)
+        fwd(i)
+        ev[i][1].record(stream)
+        back(i)
+        ev[i][2].record(stream)
+    torch.cuda.synchronize()
+    ctx.check_status()
+    f_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    b_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    ctx.close()
+    peaks = _peaks()
+    bwd_tflops = 2.0 * gemm_flops(w) / (b_ms * 1e-3) / 1e12
+    return {"fwd_ms": f_ms, "bwd_ms": b_ms, "bwd_over_fwd": b_ms / f_ms, "steps": steps,
+            "bwd_layer_tflops": bwd_tflops, "bwd_frac_of_sustained_peak": bwd_tflops / peaks["bf16_tflops_sustained"],
+            "note": "backward = combine bwd + dgrad GEMMs (fused SwiGLU derivative) + 4 transposes + 3 weight-gradient "
+                    "GEMMs (fp32 accumulate into dW) + dispatch bwd; TFLOP/s counts 12*d*f per slot over the whole "
+                    "backward time; row_align = 128"}
 
 
 def plan_sensitivity(w, dyn, policy=1, mask="reactive", split=0, n_mb=8):
@@ -437,6 +489,8 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
             "cpu_baseline": cpu, "stage_us": stage_us, "straggler": strag,
         }
+        if getattr(args, "backward_result", None):
+            line["backward"] = args.backward_result
         if args.phase2:   # Phase-2 weight copies on the copy engines, overlapped with the static GEMM
             line["phase2"] = {
                 "copy_bytes_per_step": stage_us["phase2_copy_bytes"],
@@ -498,6 +552,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-sample-tokens", type=int, default=1024)
     ap.add_argument("--no-straggler", action="store_true")
+    ap.add_argument("--backward", action="store_true", help="also time forward + backward (weight gradients included)")
     ap.add_argument("--phase2", action="store_true",
                     help="really copy migrated experts' weights into the receive buffer (copy engines) during the static GEMM")
     ap.add_argument("--quick", action="store_true",
