@@ -109,6 +109,17 @@ __device__ __forceinline__ Coord tile_coord(const Tail* t, const BwdParams& p, i
   return c;
 }
 
+// Shared-memory descriptor of an MN-major operand tile staged as 64-element (128-byte) wide boxes of
+// 64 K rows each, 128-byte swizzled: consecutive K rows are 128 bytes apart, groups of 8 K rows
+// 1024 bytes (stride byte offset), consecutive 64-element chunks along M or N one box = 8192 bytes
+// (leading byte offset) apart.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor as make_idesc, with both operands MN-major (bits 15 and 16).
+__device__ __forceinline__ uint32_t make_idesc_mn(int m, int n) { return make_idesc(m, n) | (1u << 15) | (1u << 16); }
+
 __device__ __forceinline__ float sigmoid_f(float a) { return __fdividef(1.f, 1.f + __expf(-a)); }
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
@@ -224,11 +235,13 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const uint32_t sb = sa + kABytes;
           mbar_expect_tx(full, stage_tx);
           if (KIND == KIND_WG) {
-            // K runs along the expert's rows (inner dimension of the transposed activations)
+            // K runs along the expert's rows: both operands are read as they lie in memory (row = K,
+            // columns = M resp. N contiguous), in boxes of 64 columns x 64 rows
             const int k0 = c.row0 + kb * BK;
-            tma_load_2d(sa, &tm_a, full, k0, c.mt * BM);
-            tma_load_2d(sb, &tm_b0, full, k0, c.nt * 2 * p.bn);
-            tma_load_2d(sb + b_half_bytes, &tm_b0, full, k0, c.nt * 2 * p.bn + p.bn);
+            tma_load_2d(sa, &tm_a, full, c.mt * BM, k0);
+            tma_load_2d(sa + 8192, &tm_a, full, c.mt * BM + 64, k0);
+            for (int j = 0; j < 2 * p.bn / 64; ++j)
+              tma_load_2d(sb + j * 8192, &tm_b0, full, c.nt * 2 * p.bn + 64 * j, k0);
           } else {
             const CUtensorMap* mb = (KIND == KIND_DX && kb >= p.k_switch) ? &tm_b1 : &tm_b0;
             const int kb_b = (KIND == KIND_DX && kb >= p.k_switch) ? kb - p.k_switch : kb;
@@ -247,7 +260,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   } else if (warp == 1) {
     // ---- MMA issuer -------------------------------------------------------------------------
     if (lane == 0) {
-      const uint32_t idesc = make_idesc(BM, 2 * p.bn);
+      const uint32_t idesc = KIND == KIND_WG ? make_idesc_mn(BM, 2 * p.bn) : make_idesc(BM, 2 * p.bn);
       int stage = 0, as = 0;
       uint32_t phase = 0, aphase = 0;
       bool ok = true;
@@ -260,11 +273,19 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (!(ok = mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status))) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
-          const uint64_t da = make_smem_desc(sa);
-          const uint64_t db = make_smem_desc(sa + kABytes);
+          if (KIND == KIND_WG) {
+            const uint64_t da = make_smem_desc_mn(sa);
+            const uint64_t db = make_smem_desc_mn(sa + kABytes);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+            for (int k = 0; k < BK / UMMA_K; ++k)    // 16 K rows of 128 bytes per step
+              umma_bf16(d_tmem, da + (uint64_t)(k * 128), db + (uint64_t)(k * 128), idesc, (uint32_t)((kb | k) != 0));
+          } else {
+            const uint64_t da = make_smem_desc(sa);
+            const uint64_t db = make_smem_desc(sa + kABytes);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+          }
           umma_commit(smem_u32(&tail->empty[stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -463,6 +484,20 @@ k_combine_bwd(const uint4* __restrict__ d_out, const uint4* __restrict__ y_perm,
   }
 }
 
+// Zero the rows that pad each expert's segment to a multiple of 128 rows in up to three row-major
+// buffers (blockIdx.y picks one): the weight gradients contract over whole 64-row blocks of a segment,
+// and the GEMM epilogues that produce these buffers write the valid rows only.
+struct PadBufs { uint4* buf[3]; int chunks[3]; };
+__global__ void __launch_bounds__(256)
+k_zero_pad_rows(const feplb_group* __restrict__ table, PadBufs b) {
+  const feplb_group g = table[blockIdx.x];
+  const int chunks = b.chunks[blockIdx.y];
+  const int64_t r0 = (int64_t)g.row_start + g.rows, r1 = (r0 + 127) / 128 * 128;
+  uint4* p = b.buf[blockIdx.y] + r0 * chunks;
+  const int64_t n = (r1 - r0) * chunks;
+  for (int64_t i = threadIdx.x; i < n; i += 256) p[i] = make_uint4(0, 0, 0, 0);
+}
+
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -577,31 +612,28 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   ++*n_launch;
   if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DX>");
   if (!a.dw1) return FEPLB_OK;
-  // ---- weight gradients: contraction over each expert's rows, on transposed activations -----------------
-  const int64_t ld_t = a.ld_t;     // row pitch of the transposed scratch (>= s_cap, multiple of 64)
-  char* tbuf = (char*)a.t_scratch;
-  void* xt = tbuf;                                                   // [d, ld_t]
-  void* ht = tbuf + (size_t)d * ld_t * 2;                            // [f, ld_t]
-  void* dyt = tbuf + (size_t)(d + f) * ld_t * 2;                     // [d, ld_t]
-  void* dabt = tbuf + (size_t)(2 * d + f) * ld_t * 2;                // [2f, ld_t]
-  const int rows = (int)a.s_cap;
-  e = transpose(a.x_perm, xt, rows, d, d, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
-  if (e == cudaSuccess) e = transpose(a.h, ht, rows, f, f, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
-  if (e == cudaSuccess) e = transpose(a.d_y_perm, dyt, rows, d, d, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
-  if (e == cudaSuccess) e = transpose(a.d_ab, dabt, rows, 2 * f, 2 * f, ld_t, 1, 0, 0, st, n_launch, a.row_to_token);
-  if (e != cudaSuccess) return fail_cuda("k_transpose_bf16");
+  // ---- weight gradients: contraction over each expert's rows, operands read as they lie (MN-major) ------
   // dW2[e] [d, f] = dY_e^T H_e;   dW1[e] [f, d] = dA_e^T X_e;   dW3[e] [f, d] = dB_e^T X_e
-  struct WG { const void* at; int m_total; const void* bt; int n_total; float* out; };
+  PadBufs pb;
+  pb.buf[0] = (uint4*)a.h; pb.chunks[0] = f / 8;
+  pb.buf[1] = (uint4*)a.d_y_perm; pb.chunks[1] = d / 8;
+  pb.buf[2] = (uint4*)a.d_ab; pb.chunks[2] = 2 * f / 8;
+  k_zero_pad_rows<<<dim3(a.E, 3), 256, 0, st>>>(a.expert_table, pb);
+  ++*n_launch;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda("k_zero_pad_rows");
+  struct WG { const void* p; int m_total; int ld_p; const void* q; int n_total; float* out; };
   const WG jobs[3] = {
-      {dyt, d, ht, f, a.dw2},
-      {dabt, f, xt, d, a.dw1},
-      {(const char*)dabt + (size_t)f * ld_t * 2, f, xt, d, a.dw3},
+      {a.d_y_perm, d, d, a.h, f, a.dw2},
+      {a.d_ab, f, 2 * f, a.x_perm, d, a.dw1},
+      {(const char*)a.d_ab + (size_t)f * 2, f, 2 * f, a.x_perm, d, a.dw3},
   };
   for (const WG& j : jobs) {
     const int bn = (j.n_total % 256 == 0) ? 128 : 64;
     CUtensorMap tm_at, tm_bt;
-    if (!make_tmap(&tm_at, j.at, (uint64_t)j.m_total, (uint64_t)a.s_cap, (uint64_t)ld_t, BM) ||
-        !make_tmap(&tm_bt, j.bt, (uint64_t)j.n_total, (uint64_t)a.s_cap, (uint64_t)ld_t, bn)) {
+    // boxes of 64 columns (128 bytes, the swizzle span) x 64 rows (one K block)
+    if (!make_tmap(&tm_at, j.p, (uint64_t)a.s_cap, (uint64_t)j.m_total, (uint64_t)j.ld_p, BK) ||
+        !make_tmap(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, BK)) {
       snprintf(err, errn, "cuTensorMapEncodeTiled failed (weight gradient)");
       return FEPLB_E_CUDA;
     }
