@@ -375,7 +375,7 @@ def measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, steps):
     bwd_tflops = 2.0 * gemm_flops(w) / (b_ms * 1e-3) / 1e12
     return {"fwd_ms": f_ms, "bwd_ms": b_ms, "bwd_over_fwd": b_ms / f_ms, "steps": steps,
             "bwd_layer_tflops": bwd_tflops, "bwd_frac_of_sustained_peak": bwd_tflops / peaks["bf16_tflops_sustained"],
-            "note": "backward = combine bwd + dgrad GEMMs (fused SwiGLU derivative) + 4 transposes + 3 weight-gradient "
+            "note": "backward = combine bwd + dgrad GEMMs (fused SwiGLU derivative) + 3 weight-gradient "
                     "GEMMs (fp32 accumulate into dW) + dispatch bwd; TFLOP/s counts 12*d*f per slot over the whole "
                     "backward time; row_align = 128"}
 

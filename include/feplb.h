@@ -251,8 +251,6 @@ int feplb_combine(feplb_ctx* ctx, const void* y_perm, const int32_t* slot_to_row
  * feplb_moe_forward on this context also stores the pre-activations a = x W1[e] (columns [0,f))
  * and b = x W3[e] (columns [f,2f)) of every row, which the backward pass needs.  NULL turns it off. */
 int feplb_set_preact_buffer(feplb_ctx* ctx, void* ab);
-/* Bytes of the t_scratch argument below: transposed activations, (2d + 3f) x round_up(S_cap, 64) bf16. */
-size_t feplb_bwd_scratch_bytes(const feplb_config* cfg);
 /* Transposed copies of the expert weights, needed by the activation gradients (their contractions
  * run over the weights' slow dimension): w1t, w3t dev bf16 [E, d, f]; w2t dev bf16 [E, f, d]. */
 int feplb_transpose_weights(feplb_ctx* ctx, const void* w1, const void* w3, const void* w2,
@@ -270,22 +268,24 @@ int feplb_combine_bwd(feplb_ctx* ctx, const void* d_out, const void* y_perm, con
  * row count of each expert's segment), accumulated over each expert's rows in fp32:
  *   dW2[e] = d_y_e^T H_e,  dW1[e] = dA_e^T X_e,  dW3[e] = dB_e^T X_e   (overwritten, or added to if accumulate != 0;
  *   experts without rows get zeros / stay unchanged).
- * Weight gradients need cfg.row_align = 128 and t_scratch (dev, feplb_bwd_scratch_bytes).
- * ab_saved: the buffer of feplb_set_preact_buffer; h: the forward's h_scratch. */
-int feplb_expert_ffn_bwd(feplb_ctx* ctx, const void* x_perm, const void* ab_saved, const void* h,
-                         const void* d_y_perm, const void* w1t, const void* w3t, const void* w2t,
+ * Weight gradients need cfg.row_align = 128: the contraction runs over whole 64-row blocks of an
+ * expert's segment, read in place, so the call first writes zeros to the padding rows (from the
+ * expert's row count up to the next multiple of 128) of h, d_y_perm and d_ab; x_perm's are zero
+ * already (feplb_dispatch).  ab_saved: the buffer of feplb_set_preact_buffer; h: the forward's h_scratch. */
+int feplb_expert_ffn_bwd(feplb_ctx* ctx, const void* x_perm, const void* ab_saved, void* h,
+                         void* d_y_perm, const void* w1t, const void* w3t, const void* w2t,
                          const feplb_group* groups, int32_t n_groups, int32_t which,
-                         const feplb_group* expert_table, const int32_t* row_to_token, void* d_ab,
+                         const feplb_group* expert_table, void* d_ab,
                          void* d_x_perm, float* dw1, float* dw3, float* dw2, int32_t accumulate,
-                         void* t_scratch, void* stream);
+                         void* stream);
 /* Backward of feplb_dispatch: d_x[t,:] = sum_k d_x_perm[slot_to_row[t,k],:] (fp32 sum, bf16 out). */
 int feplb_dispatch_bwd(feplb_ctx* ctx, const void* d_x_perm, const int32_t* slot_to_row, void* d_x, void* stream);
 /* The three steps above for the micro-batch whose feplb_moe_forward ran last on this context (its
  * expert table is reused): d_out -> d_x [T,d], d_gates [T,K], and the weight gradients (or NULLs). */
 int feplb_moe_backward(feplb_ctx* ctx, const void* d_out, const float* gates, const void* w1t, const void* w3t,
-                       const void* w2t, const void* x_perm, const void* ab_saved, const void* h,
-                       const void* y_perm, const int32_t* slot_to_row, const int32_t* row_to_token,
-                       void* d_y_perm, void* d_ab, void* d_x_perm, void* t_scratch, void* d_x, float* d_gates,
+                       const void* w2t, const void* x_perm, const void* ab_saved, void* h,
+                       const void* y_perm, const int32_t* slot_to_row,
+                       void* d_y_perm, void* d_ab, void* d_x_perm, void* d_x, float* d_gates,
                        float* dw1, float* dw3, float* dw2, int32_t accumulate, void* stream);
 
 /* ---- planner thread (Section 2.3: CPU balancer on a dedicated thread) ---------------------- */

@@ -791,13 +791,6 @@ extern "C" int feplb_set_preact_buffer(feplb_ctx* c, void* ab) {
   return FEPLB_OK;
 }
 
-extern "C" size_t feplb_bwd_scratch_bytes(const feplb_config* cfg) {
-  const size_t cap = feplb_s_pad(cfg);
-  if (!cap) return 0;
-  const size_t ld_t = (cap + 63) / 64 * 64;
-  return (size_t)(2 * cfg->d + 3 * cfg->f) * ld_t * 2;
-}
-
 extern "C" int feplb_transpose_weights(feplb_ctx* c, const void* w1, const void* w3, const void* w2, void* w1t, void* w3t,
                                        void* w2t, void* stream) {
   if (!c) return FEPLB_E_INVALID;
@@ -830,12 +823,12 @@ extern "C" int feplb_dispatch_bwd(feplb_ctx* c, const void* d_x_perm, const int3
   return FEPLB_OK;
 }
 
-extern "C" int feplb_expert_ffn_bwd(feplb_ctx* c, const void* x_perm, const void* ab_saved, const void* h,
-                                    const void* d_y_perm, const void* w1t, const void* w3t, const void* w2t,
+extern "C" int feplb_expert_ffn_bwd(feplb_ctx* c, const void* x_perm, const void* ab_saved, void* h,
+                                    void* d_y_perm, const void* w1t, const void* w3t, const void* w2t,
                                     const feplb_group* groups, int32_t n_groups, int32_t which,
-                                    const feplb_group* expert_table, const int32_t* row_to_token, void* d_ab,
+                                    const feplb_group* expert_table, void* d_ab,
                                     void* d_x_perm, float* dw1, float* dw3, float* dw2, int32_t accumulate,
-                                    void* t_scratch, void* stream) {
+                                    void* stream) {
   if (!c) return FEPLB_E_INVALID;
   if (n_groups < 0 || n_groups > FEPLB_MAX_GROUPS) return fail(c, FEPLB_E_INVALID, "expert_ffn_bwd: n_groups out of range");
   if (n_groups == 0 || c->s_cap == 0) return FEPLB_OK;
@@ -844,8 +837,8 @@ extern "C" int feplb_expert_ffn_bwd(feplb_ctx* c, const void* x_perm, const void
   if (!groups) return fail(c, FEPLB_E_INVALID, "expert_ffn_bwd: null group table");
   const bool want_w = dw1 || dw3 || dw2;
   if (want_w) {
-    if (!dw1 || !dw3 || !dw2 || !expert_table || !row_to_token || !t_scratch)
-      return fail(c, FEPLB_E_INVALID, "expert_ffn_bwd: weight gradients need dw1, dw3, dw2, expert_table, row_to_token, t_scratch");
+    if (!dw1 || !dw3 || !dw2 || !expert_table)
+      return fail(c, FEPLB_E_INVALID, "expert_ffn_bwd: weight gradients need dw1, dw3, dw2 and expert_table");
     if (c->cfg.row_align != 128)
       return fail(c, FEPLB_E_INVALID, "expert_ffn_bwd: weight gradients need row_align = 128 (an expert's rows are the K range)");
   }
@@ -853,26 +846,25 @@ extern "C" int feplb_expert_ffn_bwd(feplb_ctx* c, const void* x_perm, const void
   a.x_perm = x_perm; a.ab_saved = ab_saved; a.h = h; a.d_y_perm = d_y_perm;
   a.w1t = w1t; a.w3t = w3t; a.w2t = w2t;
   a.groups = groups; a.n_groups = n_groups; a.which = which;
-  a.expert_table = expert_table; a.row_to_token = row_to_token;
+  a.expert_table = expert_table;
   a.d_ab = d_ab; a.d_x_perm = d_x_perm;
   a.dw1 = want_w ? dw1 : nullptr; a.dw3 = dw3; a.dw2 = dw2; a.accumulate = accumulate != 0;
-  a.t_scratch = t_scratch; a.ld_t = ((int64_t)c->s_cap + 63) / 64 * 64;
   a.E = c->cfg.E; a.d = c->cfg.d; a.f = c->cfg.f; a.s_cap = (int64_t)c->s_cap;
   a.status = c->d_status; a.num_sms = c->num_sms;
   return feplb_launch_expert_ffn_bwd(a, (cudaStream_t)stream, &c->launches, c->err, sizeof(c->err));
 }
 
 extern "C" int feplb_moe_backward(feplb_ctx* c, const void* d_out, const float* gates, const void* w1t, const void* w3t,
-                                  const void* w2t, const void* x_perm, const void* ab_saved, const void* h,
-                                  const void* y_perm, const int32_t* slot_to_row, const int32_t* row_to_token,
-                                  void* d_y_perm, void* d_ab, void* d_x_perm, void* t_scratch, void* d_x, float* d_gates,
+                                  const void* w2t, const void* x_perm, const void* ab_saved, void* h,
+                                  const void* y_perm, const int32_t* slot_to_row,
+                                  void* d_y_perm, void* d_ab, void* d_x_perm, void* d_x, float* d_gates,
                                   float* dw1, float* dw3, float* dw2, int32_t accumulate, void* stream) {
   if (!c) return FEPLB_E_INVALID;
   int rc = feplb_combine_bwd(c, d_out, y_perm, slot_to_row, gates, d_y_perm, d_gates, stream);
   if (rc != FEPLB_OK) return rc;
   // every expert's rows in one table: the home table of the forward pass that ran last on this context
   rc = feplb_expert_ffn_bwd(c, x_perm, ab_saved, h, d_y_perm, w1t, w3t, w2t, c->d_home_groups, c->cfg.E, FEPLB_FFN_ALL,
-                            c->d_home_groups, row_to_token, d_ab, d_x_perm, dw1, dw3, dw2, accumulate, t_scratch, stream);
+                            c->d_home_groups, d_ab, d_x_perm, dw1, dw3, dw2, accumulate, stream);
   if (rc != FEPLB_OK) return rc;
   return feplb_dispatch_bwd(c, d_x_perm, slot_to_row, d_x, stream);
 }

@@ -1,14 +1,15 @@
 // Backward pass of the grouped SwiGLU expert FFN on sm_100a (the paper reports backward layer times
 // in Table 2 but does not describe the pass; this is the derivative of the forward definition,
-// computed over the same groups).  One warp-specialised tcgen05 kernel in three kinds, all with
-// K-major operands staged by TMA (weights and activations are transposed beforehand where the
-// contraction runs over their slow dimension):
+// computed over the same groups).  One warp-specialised tcgen05 kernel in three kinds, operands
+// staged by TMA.  DH and DX take K-major operands (the weights are transposed once per weight
+// update, their contraction runs over the forward layout's slow dimension); WG takes MN-major
+// operands, i.e. the row-major activations as they lie, the contraction running over rows:
 //   DH: dH = dY W2 (A = dY rows, B = W2^T tiles), epilogue applies the SwiGLU derivative with the
 //       saved pre-activations:  dA = dH * b * silu'(a),  dB = dH * silu(a)  -> dAB [rows, 2f]
 //   DX: dX = dA W1^T + dB W3^T as ONE contraction over K = 2f ([dA|dB] against W1^T then W3^T)
 //   WG: weight gradients, one (expert, M tile, N tile) per tile with the contraction running over
-//       that expert's rows:  dW[e] = P_e^T Q_e  (fp32 out, optionally accumulated), operands are
-//       the transposed activations P^T [M, rows], Q^T [N, rows]
+//       that expert's rows:  dW[e] = P_e^T Q_e  (fp32 out, optionally accumulated), P [rows, M] and
+//       Q [rows, N] read in boxes of 64 columns x 64 rows, padding rows zeroed beforehand
 // Pipeline as in the forward kernel: warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps
 // 2..5 epilogue; 4-stage ring of 48 KiB; two TMEM accumulators; every mbarrier wait bounded.
 #include <cuda.h>
@@ -37,6 +38,12 @@ constexpr int kStageBytes = kABytes + kBBytesMax;
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kEpiStageBytes = 32 * 128;
+// The weight-gradient kind gives up one ring stage for output staging: each epilogue warp owns
+// kWgBufs buffers of 32 rows x 32 fp32 (4 KiB, 128-byte swizzled) that TMA stores or reduce-adds
+// drain to dW while the warp fills the next one.
+constexpr int kWgStages = 3;
+constexpr int kWgBufs = 4;
+static_assert(kWgBufs * kEpiWarps * kEpiStageBytes <= kABytes + kBBytesMax + kEpiWarps * kEpiStageBytes, "staging fits the freed stage");
 
 struct Tail {
   unsigned long long full[kStages];
@@ -147,14 +154,29 @@ __device__ __forceinline__ void staged_store(uint32_t stg, const uint32_t* packe
   __syncwarp();
 }
 
+// TMA store / reduce-add of one staged 32 x 32 fp32 box to dW[e] (tensor map over [E, M, N]).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(m), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* m, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(m), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 template <int KIND>
 __global__ void __launch_bounds__(kThreads, 1)
 k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
-               const __grid_constant__ CUtensorMap tm_b1, const BwdParams p) {
+               const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_out, const BwdParams p) {
+  constexpr int NS = KIND == KIND_WG ? kWgStages : kStages;      // ring stages
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* epi_smem = smem + (size_t)kStages * kStageBytes;
-  Tail* tail = reinterpret_cast<Tail*>(epi_smem + (size_t)kEpiWarps * kEpiStageBytes);
+  uint8_t* epi_smem = smem + (size_t)NS * kStageBytes;
+  Tail* tail = reinterpret_cast<Tail*>(smem + (size_t)kStages * kStageBytes + (size_t)kEpiWarps * kEpiStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &tail->abort_flag;
 
@@ -162,7 +184,8 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     prefetch_tmap(&tm_a);
     prefetch_tmap(&tm_b0);
     prefetch_tmap(&tm_b1);
-    for (int s = 0; s < kStages; ++s) {
+    if (KIND == KIND_WG) prefetch_tmap(&tm_out);
+    for (int s = 0; s < NS; ++s) {
       mbar_init(smem_u32(&tail->full[s]), 1);
       mbar_init(smem_u32(&tail->empty[s]), 1);
     }
@@ -250,7 +273,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             tma_load_2d(sb, mb, full, kb_b * BK, brow);
             tma_load_2d(sb + b_half_bytes, mb, full, kb_b * BK, brow + p.bn);
           }
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
@@ -287,7 +310,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
               umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
           }
           umma_commit(smem_u32(&tail->empty[stage]));
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         if (c.kblocks > 0) umma_commit(smem_u32(&tail->tmem_full[as]));
@@ -298,7 +321,8 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   } else {
     // ---- epilogue -----------------------------------------------------------------------------
     const int q = warp & 3;
-    const uint32_t stg = smem_u32(epi_smem + (size_t)(warp - 2) * kEpiStageBytes);
+    const uint32_t stg = smem_u32(epi_smem + (size_t)(warp - 2) * kEpiStageBytes * (KIND == KIND_WG ? kWgBufs : 1));
+    int wg_buf = 0;
     int as = 0;
     uint32_t aphase = 0;
     bool ok = true;
@@ -311,10 +335,14 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * kAccCols);
       const int out_cols = 2 * p.bn;
       if (KIND == KIND_WG) {
-        // fp32 tile of dW[e]: thread = row of the M tile, 32 consecutive columns = one 128-byte line
-        const int m = c.mt * BM + q * 32 + lane;
-        float* orow = p.wout + ((int64_t)c.expert * p.m_total + m) * p.n_total + (int64_t)c.nt * out_cols;
+        // fp32 tile of dW[e]: this warp's 32 rows, 32 columns at a time: TMEM -> registers ->
+        // swizzled staging buffer -> one TMA store (or reduce-add into dW) of the 32 x 32 box.
+        // An expert without rows adds nothing; without accumulation it gets zeros.
+        const int m0 = c.mt * BM + q * 32;
+        const bool emit = m0 < p.m_total && !(c.kblocks == 0 && p.accumulate);
         for (int col = 0; col < out_cols; col += 32) {
+          const int n0 = c.nt * out_cols + col;
+          if (!emit || n0 >= p.n_total) continue;     // warp-uniform; M and N are multiples of 32
           uint32_t a[32];
           if (c.kblocks > 0) {
             tmem_ld32(taddr + (uint32_t)col, a);
@@ -323,20 +351,23 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
             for (int i = 0; i < 32; ++i) a[i] = 0u;
           }
-          const int n0 = c.nt * out_cols + col;
-          if (m < p.m_total && n0 < p.n_total) {      // n_total is a multiple of 32
-            float4* dst = reinterpret_cast<float4*>(orow + col);
+          const uint32_t buf = stg + (uint32_t)(wg_buf * kEpiStageBytes);
+          if (lane == 0) bulk_wait_read<kWgBufs - 1>();     // the store that read this buffer kWgBufs boxes ago
+          __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float4 v = make_float4(__uint_as_float(a[4 * i]), __uint_as_float(a[4 * i + 1]),
-                                     __uint_as_float(a[4 * i + 2]), __uint_as_float(a[4 * i + 3]));
-              if (p.accumulate) {
-                const float4 o = dst[i];
-                v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-              }
-              dst[i] = v;
-            }
+          for (int j = 0; j < 8; ++j) {
+            const uint32_t addr = buf + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a[4 * j]), "r"(a[4 * j + 1]),
+                         "r"(a[4 * j + 2]), "r"(a[4 * j + 3]) : "memory");
           }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (p.accumulate) tma_reduce_add_3d(&tm_out, buf, n0, m0, c.expert);
+            else tma_store_3d(&tm_out, buf, n0, m0, c.expert);
+            bulk_commit();
+          }
+          if (++wg_buf == kWgBufs) wg_buf = 0;
         }
       } else {
         const int row_off = q * 32;
@@ -397,6 +428,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[as]));
       if (++as == kAccStages) { as = 0; aphase ^= 1u; }
     }
+    if (KIND == KIND_WG && lane == 0) bulk_wait_read<0>();      // staging must outlive the stores that read it
   }
 
   tc_fence_before();
@@ -410,14 +442,11 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
 // ---- bandwidth kernels of the backward pass ---------------------------------------------------
 
-// dst[c, r] = src[r, c] for a batch of bf16 matrices (32 x 32 tiles through shared memory).  With
-// row_token != nullptr, source rows that hold no token (row_token[r] < 0: the padding at the end
-// of an expert's segment, never written by the masked stores of the GEMMs) are transposed as
-// zeros, so that they add nothing to a contraction over rows.
+// dst[c, r] = src[r, c] for a batch of bf16 matrices (32 x 32 tiles through shared memory); used
+// once per weight update for the transposed weight copies, not per micro-batch.
 __global__ void __launch_bounds__(256)
 k_transpose_bf16(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows, int cols,
-                 int64_t ld_src, int64_t ld_dst, int64_t batch_src, int64_t batch_dst,
-                 const int32_t* __restrict__ row_token) {
+                 int64_t ld_src, int64_t ld_dst, int64_t batch_src, int64_t batch_dst) {
   __shared__ __nv_bfloat16 t[32][34];
   src += (int64_t)blockIdx.z * batch_src;
   dst += (int64_t)blockIdx.z * batch_dst;
@@ -426,7 +455,7 @@ k_transpose_bf16(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restric
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = r0 + ty + 8 * i, c = c0 + tx;
-    const bool live = r < rows && c < cols && (row_token == nullptr || row_token[r] >= 0);
+    const bool live = r < rows && c < cols;
     t[ty + 8 * i][tx] = live ? src[(int64_t)r * ld_src + c] : __float2bfloat16(0.f);
   }
   __syncthreads();
@@ -527,26 +556,38 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 [E, M, N] as a 3-d map with boxes of 32 x 32 x 1, 128-byte swizzled (the epilogue's staging layout);
+// a box never crosses into the next expert's matrix.
+bool make_tmap_out(CUtensorMap* m, float* base, uint64_t E, uint64_t M, uint64_t N) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {N, M, E};
+  cuuint64_t strides[2] = {N * 4, M * N * 4};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int KIND>
-cudaError_t launch_kind(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const BwdParams& p,
-                        int grid, cudaStream_t st) {
+cudaError_t launch_kind(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tout,
+                        const BwdParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(k_ffn_bwd_gemm<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  k_ffn_bwd_gemm<KIND><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, p);
+  k_ffn_bwd_gemm<KIND><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, tout, p);
   return cudaGetLastError();
 }
 
 cudaError_t transpose(const void* src, void* dst, int rows, int cols, int64_t ld_src, int64_t ld_dst, int batch,
-                      int64_t batch_src, int64_t batch_dst, cudaStream_t st, int64_t* n_launch,
-                      const int32_t* row_token = nullptr) {
+                      int64_t batch_src, int64_t batch_dst, cudaStream_t st, int64_t* n_launch) {
   if (rows == 0 || cols == 0 || batch == 0) return cudaSuccess;
   dim3 grid((cols + 31) / 32, (rows + 31) / 32, batch);
   k_transpose_bf16<<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (__nv_bfloat16*)dst, rows, cols, ld_src, ld_dst,
-                                         batch_src, batch_dst, row_token);
+                                         batch_src, batch_dst);
   ++*n_launch;
   return cudaGetLastError();
 }
@@ -601,14 +642,14 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   BwdParams ph = p;
   ph.n_tiles_n = (f + 2 * bn_h - 1) / (2 * bn_h); ph.n_limit = f; ph.num_k_blocks = d / BK; ph.b_rows_per_expert = f; ph.bn = bn_h;
   ph.out = (__nv_bfloat16*)a.d_ab; ph.ld_out = 2 * f; ph.ab = (const __nv_bfloat16*)a.ab_saved; ph.f = f;
-  e = launch_kind<KIND_DH>(tm_dy, tm_w2t, tm_w2t, ph, a.num_sms, st);
+  e = launch_kind<KIND_DH>(tm_dy, tm_w2t, tm_w2t, tm_dy, ph, a.num_sms, st);
   ++*n_launch;
   if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DH>");
   // ---- dX = [dA | dB] [W1^T ; W3^T] ------------------------------------------------------------------
   BwdParams px = p;
   px.n_tiles_n = d / (2 * bn_x); px.n_limit = d; px.num_k_blocks = 2 * f / BK; px.k_switch = f / BK; px.b_rows_per_expert = d; px.bn = bn_x;
   px.out = (__nv_bfloat16*)a.d_x_perm; px.ld_out = d;
-  e = launch_kind<KIND_DX>(tm_dab, tm_w1t, tm_w3t, px, a.num_sms, st);
+  e = launch_kind<KIND_DX>(tm_dab, tm_w1t, tm_w3t, tm_dab, px, a.num_sms, st);
   ++*n_launch;
   if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DX>");
   if (!a.dw1) return FEPLB_OK;
@@ -630,10 +671,11 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   };
   for (const WG& j : jobs) {
     const int bn = (j.n_total % 256 == 0) ? 128 : 64;
-    CUtensorMap tm_at, tm_bt;
+    CUtensorMap tm_at, tm_bt, tm_o;
     // boxes of 64 columns (128 bytes, the swizzle span) x 64 rows (one K block)
     if (!make_tmap(&tm_at, j.p, (uint64_t)a.s_cap, (uint64_t)j.m_total, (uint64_t)j.ld_p, BK) ||
-        !make_tmap(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, BK)) {
+        !make_tmap(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, BK) ||
+        !make_tmap_out(&tm_o, j.out, (uint64_t)a.E, (uint64_t)j.m_total, (uint64_t)j.n_total)) {
       snprintf(err, errn, "cuTensorMapEncodeTiled failed (weight gradient)");
       return FEPLB_E_CUDA;
     }
@@ -641,7 +683,7 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
     pw.groups = a.expert_table; pw.n_groups = a.E; pw.which = FEPLB_FFN_ALL;
     pw.bn = bn; pw.n_tiles_n = (j.n_total + 2 * bn - 1) / (2 * bn); pw.m_tiles = (j.m_total + BM - 1) / BM;
     pw.m_total = j.m_total; pw.n_total = j.n_total; pw.wout = j.out; pw.accumulate = a.accumulate;
-    e = launch_kind<KIND_WG>(tm_at, tm_bt, tm_bt, pw, a.num_sms, st);
+    e = launch_kind<KIND_WG>(tm_at, tm_bt, tm_bt, tm_o, pw, a.num_sms, st);
     ++*n_launch;
     if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<WG>");
   }

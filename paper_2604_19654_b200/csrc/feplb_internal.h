@@ -76,14 +76,12 @@ cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limi
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
 // ---- backward pass ---------------------------------------------------------------------------
 struct feplb_bwd_args {
-  const void* x_perm; const void* ab_saved; const void* h; const void* d_y_perm;
+  const void* x_perm; const void* ab_saved; void* h; void* d_y_perm;   // padding rows of h, d_y_perm, d_ab get zeros
   const void* w1t; const void* w3t; const void* w2t;        // [E,d,f], [E,d,f], [E,f,d]
   const feplb_group* groups; int n_groups; int which;
   const feplb_group* expert_table;                          // E entries {e, first row, rows}: the K ranges of the weight gradients
-  const int32_t* row_to_token;
   void* d_ab; void* d_x_perm;                               // [s_cap, 2f], [s_cap, d]
   float* dw1; float* dw3; float* dw2; int accumulate;       // fp32 [E,f,d], [E,f,d], [E,d,f]; dw1 == nullptr: skip
-  void* t_scratch; int64_t ld_t;                            // transposed activations: (2d + 3f) rows of ld_t bf16
   int E, d, f; int64_t s_cap;
   uint32_t* status; int num_sms;
 };

@@ -98,12 +98,11 @@ def lib() -> C.CDLL:
             "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
             "feplb_timeline_totals": (C.c_int, [vp, C.POINTER(Timeline), C.POINTER(i64), i32]),
             "feplb_set_preact_buffer": (C.c_int, [vp, vp]),
-            "feplb_bwd_scratch_bytes": (C.c_size_t, [C.POINTER(Config)]),
             "feplb_transpose_weights": (C.c_int, [vp] * 8),
             "feplb_combine_bwd": (C.c_int, [vp] * 8),
-            "feplb_expert_ffn_bwd": (C.c_int, [vp] * 9 + [i32, i32] + [vp] * 7 + [i32, vp, vp]),
+            "feplb_expert_ffn_bwd": (C.c_int, [vp] * 9 + [i32, i32] + [vp] * 6 + [i32, vp]),
             "feplb_dispatch_bwd": (C.c_int, [vp] * 5),
-            "feplb_moe_backward": (C.c_int, [vp] * 21 + [i32, vp]),
+            "feplb_moe_backward": (C.c_int, [vp] * 19 + [i32, vp]),
             "feplb_set_planner_timeout": (C.c_int, [vp, i32]),
             "feplb_selftest_bounded_wait": (C.c_int, [vp, i32, vp]),
             "feplb_launch_count": (i64, [vp]),
@@ -376,13 +375,12 @@ class Context:
         self._chk(lib().feplb_combine_bwd(self._h, _ptr(d_out), _ptr(y_perm), _ptr(slot_to_row), _ptr(gates),
                                           _ptr(d_y_perm), _ptr(d_gates), self._stream(stream)), "feplb_combine_bwd")
 
-    def expert_ffn_bwd(self, x_perm, ab_saved, h, d_y_perm, w1t, w3t, w2t, groups, n_groups, expert_table, row_to_token,
-                       d_ab, d_x_perm, dw1=None, dw3=None, dw2=None, accumulate=False, t_scratch=None, which=FFN_ALL,
-                       stream=None):
+    def expert_ffn_bwd(self, x_perm, ab_saved, h, d_y_perm, w1t, w3t, w2t, groups, n_groups, expert_table,
+                       d_ab, d_x_perm, dw1=None, dw3=None, dw2=None, accumulate=False, which=FFN_ALL, stream=None):
         self._chk(lib().feplb_expert_ffn_bwd(
             self._h, _ptr(x_perm), _ptr(ab_saved), _ptr(h), _ptr(d_y_perm), _ptr(w1t), _ptr(w3t), _ptr(w2t), _ptr(groups),
-            int(n_groups), int(which), _ptr(expert_table), _ptr(row_to_token), _ptr(d_ab), _ptr(d_x_perm), _ptr(dw1),
-            _ptr(dw3), _ptr(dw2), int(bool(accumulate)), _ptr(t_scratch), self._stream(stream)), "feplb_expert_ffn_bwd")
+            int(n_groups), int(which), _ptr(expert_table), _ptr(d_ab), _ptr(d_x_perm), _ptr(dw1),
+            _ptr(dw3), _ptr(dw2), int(bool(accumulate)), self._stream(stream)), "feplb_expert_ffn_bwd")
 
     def dispatch_bwd(self, d_x_perm, slot_to_row, d_x, stream=None):
         self._chk(lib().feplb_dispatch_bwd(self._h, _ptr(d_x_perm), _ptr(slot_to_row), _ptr(d_x), self._stream(stream)),
@@ -390,11 +388,11 @@ class Context:
 
     def moe_backward(self, d_out, gates, w1t, w3t, w2t, buf, bwd, dw1=None, dw3=None, dw2=None, accumulate=False,
                      stream=None):
-        """``buf``: the forward's Buffers; ``bwd``: a BackwardBuffers (ab, d_y_perm, d_ab, d_x_perm, t_scratch, d_x, d_gates)."""
+        """``buf``: the forward's Buffers; ``bwd``: a BackwardBuffers (ab, d_y_perm, d_ab, d_x_perm, d_x, d_gates)."""
         self._chk(lib().feplb_moe_backward(
             self._h, _ptr(d_out), _ptr(gates), _ptr(w1t), _ptr(w3t), _ptr(w2t), _ptr(buf.x_perm), _ptr(bwd.ab),
-            _ptr(buf.h_scratch), _ptr(buf.y_perm), _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(bwd.d_y_perm),
-            _ptr(bwd.d_ab), _ptr(bwd.d_x_perm), _ptr(bwd.t_scratch), _ptr(bwd.d_x), _ptr(bwd.d_gates), _ptr(dw1),
+            _ptr(buf.h_scratch), _ptr(buf.y_perm), _ptr(buf.slot_to_row), _ptr(bwd.d_y_perm),
+            _ptr(bwd.d_ab), _ptr(bwd.d_x_perm), _ptr(bwd.d_x), _ptr(bwd.d_gates), _ptr(dw1),
             _ptr(dw3), _ptr(dw2), int(bool(accumulate)), self._stream(stream)), "feplb_moe_backward")
 
     def set_planner_timeout(self, timeout_ms: int):
@@ -437,7 +435,6 @@ class BackwardBuffers:
         self.d_y_perm = torch.zeros(cap, cfg.d, dtype=bf, device=device)
         self.d_ab = torch.zeros(cap, 2 * cfg.f, dtype=bf, device=device)
         self.d_x_perm = torch.zeros(cap, cfg.d, dtype=bf, device=device)
-        self.t_scratch = torch.empty(max(int(lib().feplb_bwd_scratch_bytes(C.byref(cfg))), 16), dtype=torch.uint8, device=device)
         self.d_x = torch.zeros(max(cfg.T, 1), cfg.d, dtype=bf, device=device)
         self.d_gates = torch.zeros(max(cfg.T, 1), cfg.K, dtype=torch.float32, device=device)
 
