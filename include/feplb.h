@@ -339,6 +339,15 @@ int feplb_moe_forward_host_async(feplb_ctx* ctx, int32_t slot, const void* x_hos
                                  int32_t* counts, int32_t* rank_load, void* x_perm, void* h_scratch, void* y_perm,
                                  int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
                                  feplb_plan_out* plan_copy, void* stream);
+/* Optional prefetch for feplb_moe_forward_host_async: starts the copies of a micro-batch's inputs
+ * (host, pinned) into the staging set of `slot` on the context's input stream, after the forward
+ * that last read that staging set, and returns at once.  The next feplb_moe_forward_host_async
+ * on this slot then uses what was staged and ignores its three host input pointers.  Called
+ * for micro-batch i+1 before the forward of micro-batch i, it lets the input copies run under
+ * a whole forward instead of only under its tail.  The host buffers must stay untouched until that
+ * forward's feplb_host_wait. */
+int feplb_host_stage_inputs(feplb_ctx* ctx, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
+                            const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev);
 /* Blocks until the result of the last feplb_moe_forward_host_async on `slot` is in its out_host. */
 int feplb_host_wait(feplb_ctx* ctx, int32_t slot);
 

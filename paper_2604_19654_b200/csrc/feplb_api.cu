@@ -67,6 +67,7 @@ struct feplb_ctx {
   cudaStream_t in_stream = nullptr, out_stream = nullptr;
   cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
   bool slot_used[2] = {false, false};
+  bool slot_staged[2] = {false, false};        // inputs already on their way (feplb_host_stage_inputs)
   cudaEvent_t ev_counts = nullptr, ev_plan = nullptr;
   cudaEvent_t evr[kEvRing][EV_N] = {{nullptr}};
   cudaEvent_t* ev = evr[0];        // event set of the current forward
@@ -676,6 +677,27 @@ extern "C" int feplb_moe_forward_host(feplb_ctx* c, const void* x_host, const in
   return FEPLB_OK;
 }
 
+extern "C" int feplb_host_stage_inputs(feplb_ctx* c, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
+                                       const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev) {
+  if (!c) return FEPLB_E_INVALID;
+  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "host_stage_inputs: slot must be 0 or 1");
+  if (c->slot_staged[slot]) return fail(c, FEPLB_E_STATE, "host_stage_inputs: slot %d already holds staged inputs", slot);
+  const feplb_config& g = c->cfg;
+  const size_t nx = (size_t)g.T * g.d * 2, nk = (size_t)g.T * g.K * 4;
+  if (g.T > 0 && (!x_host || !topk_ids_host || !gates_host || !x_dev || !ids_dev || !gates_dev))
+    return fail(c, FEPLB_E_INVALID, "host_stage_inputs: null pointer");
+  // the slot's device staging was last read by the forward that used this slot before
+  if (c->slot_used[slot]) CUDA_TRY(c, cudaStreamWaitEvent(c->in_stream, c->ev_done[slot], 0));
+  if (g.T > 0) {
+    CUDA_TRY(c, cudaMemcpyAsync(ids_dev, topk_ids_host, nk, cudaMemcpyHostToDevice, c->in_stream));
+    CUDA_TRY(c, cudaMemcpyAsync(gates_dev, gates_host, nk, cudaMemcpyHostToDevice, c->in_stream));
+    CUDA_TRY(c, cudaMemcpyAsync(x_dev, x_host, nx, cudaMemcpyHostToDevice, c->in_stream));
+  }
+  CUDA_TRY(c, cudaEventRecord(c->ev_in[slot], c->in_stream));
+  c->slot_staged[slot] = true;
+  return FEPLB_OK;
+}
+
 extern "C" int feplb_moe_forward_host_async(feplb_ctx* c, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
                                             const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
                                             const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,
@@ -686,17 +708,16 @@ extern "C" int feplb_moe_forward_host_async(feplb_ctx* c, int32_t slot, const vo
   if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: slot must be 0 or 1");
   cudaStream_t st = (cudaStream_t)stream;
   const feplb_config& g = c->cfg;
-  const size_t nx = (size_t)g.T * g.d * 2, nk = (size_t)g.T * g.K * 4;
-  if (g.T > 0 && (!x_host || !topk_ids_host || !gates_host || !out_host || !x_dev || !ids_dev || !gates_dev || !out_dev))
+  const size_t nx = (size_t)g.T * g.d * 2;
+  if (g.T > 0 && (!out_host || !x_dev || !ids_dev || !gates_dev || !out_dev))
     return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: null pointer");
-  // inputs: the slot's device staging was last read by the forward that used this slot before
-  if (c->slot_used[slot]) CUDA_TRY(c, cudaStreamWaitEvent(c->in_stream, c->ev_done[slot], 0));
-  if (g.T > 0) {
-    CUDA_TRY(c, cudaMemcpyAsync(ids_dev, topk_ids_host, nk, cudaMemcpyHostToDevice, c->in_stream));
-    CUDA_TRY(c, cudaMemcpyAsync(gates_dev, gates_host, nk, cudaMemcpyHostToDevice, c->in_stream));
-    CUDA_TRY(c, cudaMemcpyAsync(x_dev, x_host, nx, cudaMemcpyHostToDevice, c->in_stream));
+  if (c->slot_staged[slot]) {
+    c->slot_staged[slot] = false;        // inputs were started by feplb_host_stage_inputs; ev_in[slot] marks their end
+  } else {
+    int rc = feplb_host_stage_inputs(c, slot, x_host, topk_ids_host, gates_host, x_dev, ids_dev, gates_dev);
+    if (rc != FEPLB_OK) return rc;
+    c->slot_staged[slot] = false;
   }
-  CUDA_TRY(c, cudaEventRecord(c->ev_in[slot], c->in_stream));
   // compute: after its inputs have arrived and the slot's previous result has left out_dev
   CUDA_TRY(c, cudaStreamWaitEvent(st, c->ev_in[slot], 0));
   if (c->slot_used[slot]) CUDA_TRY(c, cudaStreamWaitEvent(st, c->ev_out[slot], 0));

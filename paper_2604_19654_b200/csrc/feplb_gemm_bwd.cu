@@ -154,6 +154,13 @@ __device__ __forceinline__ void staged_store(uint32_t stg, const uint32_t* packe
   __syncwarp();
 }
 
+// 3-d tiled TMA load (the MN-major operands: 64 columns x 64 rows x several 64-column chunks).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 // TMA store / reduce-add of one staged 32 x 32 fp32 box to dW[e] (tensor map over [E, M, N]).
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
@@ -259,12 +266,11 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           mbar_expect_tx(full, stage_tx);
           if (KIND == KIND_WG) {
             // K runs along the expert's rows: both operands are read as they lie in memory (row = K,
-            // columns = M resp. N contiguous), in boxes of 64 columns x 64 rows
+            // columns = M resp. N contiguous).  The maps see a matrix as [64-column chunk][row][64
+            // columns], so one load brings 64 rows of all the tile's chunks, 8 KiB per chunk.
             const int k0 = c.row0 + kb * BK;
-            tma_load_2d(sa, &tm_a, full, c.mt * BM, k0);
-            tma_load_2d(sa + 8192, &tm_a, full, c.mt * BM + 64, k0);
-            for (int j = 0; j < 2 * p.bn / 64; ++j)
-              tma_load_2d(sb + j * 8192, &tm_b0, full, c.nt * 2 * p.bn + 64 * j, k0);
+            tma_load_3d(sa, &tm_a, full, 0, k0, c.mt * (BM / 64));
+            tma_load_3d(sb, &tm_b0, full, 0, k0, c.nt * (2 * p.bn / 64));
           } else {
             const CUtensorMap* mb = (KIND == KIND_DX && kb >= p.k_switch) ? &tm_b1 : &tm_b0;
             const int kb_b = (KIND == KIND_DX && kb >= p.k_switch) ? kb - p.k_switch : kb;
@@ -515,7 +521,8 @@ k_combine_bwd(const uint4* __restrict__ d_out, const uint4* __restrict__ y_perm,
 
 // Zero the rows that pad each expert's segment to a multiple of 128 rows in up to three row-major
 // buffers (blockIdx.y picks one): the weight gradients contract over whole 64-row blocks of a segment,
-// and the GEMM epilogues that produce these buffers write the valid rows only.
+// and the GEMM epilogues that produce these buffers write the valid rows only.  gridDim.z blocks
+// share one (expert, buffer).
 struct PadBufs { uint4* buf[3]; int chunks[3]; };
 __global__ void __launch_bounds__(256)
 k_zero_pad_rows(const feplb_group* __restrict__ table, PadBufs b) {
@@ -524,7 +531,7 @@ k_zero_pad_rows(const feplb_group* __restrict__ table, PadBufs b) {
   const int64_t r0 = (int64_t)g.row_start + g.rows, r1 = (r0 + 127) / 128 * 128;
   uint4* p = b.buf[blockIdx.y] + r0 * chunks;
   const int64_t n = (r1 - r0) * chunks;
-  for (int64_t i = threadIdx.x; i < n; i += 256) p[i] = make_uint4(0, 0, 0, 0);
+  for (int64_t i = blockIdx.z * 256 + threadIdx.x; i < n; i += 256 * gridDim.z) p[i] = make_uint4(0, 0, 0, 0);
 }
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -552,6 +559,21 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
   cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Row-major bf16 [rows, cols] (pitch ld) as the 3-d tensor {64 columns, rows, cols/64 chunks}: a box of
+// 64 x 64 x `chunks` lands in shared memory chunk after chunk, each 64 rows of 128 bytes, 128-byte
+// swizzled: the MN-major operand layout of the weight-gradient kind.
+bool make_tmap_mn(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t chunks) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {64, rows, cols / 64};
+  cuuint64_t strides[2] = {ld * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)BK, chunks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -659,7 +681,7 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   pb.buf[0] = (uint4*)a.h; pb.chunks[0] = f / 8;
   pb.buf[1] = (uint4*)a.d_y_perm; pb.chunks[1] = d / 8;
   pb.buf[2] = (uint4*)a.d_ab; pb.chunks[2] = 2 * f / 8;
-  k_zero_pad_rows<<<dim3(a.E, 3), 256, 0, st>>>(a.expert_table, pb);
+  k_zero_pad_rows<<<dim3(a.E, 3, 8), 256, 0, st>>>(a.expert_table, pb);
   ++*n_launch;
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda("k_zero_pad_rows");
@@ -672,9 +694,8 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   for (const WG& j : jobs) {
     const int bn = (j.n_total % 256 == 0) ? 128 : 64;
     CUtensorMap tm_at, tm_bt, tm_o;
-    // boxes of 64 columns (128 bytes, the swizzle span) x 64 rows (one K block)
-    if (!make_tmap(&tm_at, j.p, (uint64_t)a.s_cap, (uint64_t)j.m_total, (uint64_t)j.ld_p, BK) ||
-        !make_tmap(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, BK) ||
+    if (!make_tmap_mn(&tm_at, j.p, (uint64_t)a.s_cap, (uint64_t)j.m_total, (uint64_t)j.ld_p, BM / 64) ||
+        !make_tmap_mn(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, 2 * bn / 64) ||
         !make_tmap_out(&tm_o, j.out, (uint64_t)a.E, (uint64_t)j.m_total, (uint64_t)j.n_total)) {
       snprintf(err, errn, "cuTensorMapEncodeTiled failed (weight gradient)");
       return FEPLB_E_CUDA;

@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
             "feplb_moe_forward_host": (C.c_int, [vp] * 20 + [C.POINTER(PlanOut), vp]),
             "feplb_moe_forward_host_async": (C.c_int, [vp, i32] + [vp] * 19 + [C.POINTER(PlanOut), vp]),
             "feplb_host_wait": (C.c_int, [vp, i32]),
+            "feplb_host_stage_inputs": (C.c_int, [vp, i32] + [vp] * 6),
             "feplb_set_timeline": (C.c_int, [vp, i32]),
             "feplb_get_timeline": (C.c_int, [vp, C.POINTER(Timeline)]),
             "feplb_timeline_totals": (C.c_int, [vp, C.POINTER(Timeline), C.POINTER(i64), i32]),
@@ -345,6 +346,11 @@ class Context:
             _ptr(buf.counts), _ptr(buf.rank_load), _ptr(buf.x_perm), _ptr(buf.h_scratch), _ptr(buf.y_perm),
             _ptr(buf.slot_to_row), _ptr(buf.row_to_token), _ptr(out_dev), _ptr(out_host), None,
             self._stream(stream)), "feplb_moe_forward_host_async")
+
+    def host_stage_inputs(self, slot, x_host, ids_host, gates_host, x_dev, ids_dev, gates_dev):
+        """Start the input copies of the next micro-batch into staging slot ``slot`` ahead of its forward."""
+        self._chk(lib().feplb_host_stage_inputs(self._h, int(slot), _ptr(x_host), _ptr(ids_host), _ptr(gates_host),
+                                                _ptr(x_dev), _ptr(ids_dev), _ptr(gates_dev)), "feplb_host_stage_inputs")
 
     def host_wait(self, slot):
         self._chk(lib().feplb_host_wait(self._h, int(slot)), "feplb_host_wait")

@@ -412,6 +412,25 @@ def test_pipelined_host_forward_matches_the_synchronous_one():
     case.ctx.check_status()
     for n in range(len(pin)):
         assert np.array_equal(outs[n].numpy(), ref[n]), n
+    # the same with the inputs of micro-batch n+1 staged ahead of the forward of micro-batch n;
+    # the forward then ignores its host input pointers (a wrong micro-batch's are passed on purpose)
+    outs2 = [torch.zeros(w.T, w.d, dtype=torch.int16).pin_memory() for _ in pin]
+    case.ctx.host_stage_inputs(0, *pin[0], x_dev[0], i_dev[0], g_dev[0])
+    with pytest.raises(F.FeplbError):
+        case.ctx.host_stage_inputs(0, *pin[0], x_dev[0], i_dev[0], g_dev[0])      # slot already staged
+    for n in range(len(pin)):
+        s = n & 1
+        if n + 1 < len(pin):
+            case.ctx.host_stage_inputs(s ^ 1, *pin[n + 1], x_dev[s ^ 1], i_dev[s ^ 1], g_dev[s ^ 1])
+        case.ctx.host_wait(s)
+        xh, ih, gh = pin[(n + 1) % len(pin)]
+        case.ctx.moe_forward_host_async(s, xh, ih, gh, x_dev[s], i_dev[s], g_dev[s], case.d_w1, case.d_w3, case.d_w2,
+                                        case.buf, o_dev[s], outs2[n])
+    case.ctx.host_wait(0)
+    case.ctx.host_wait(1)
+    case.ctx.check_status()
+    for n in range(len(pin)):
+        assert np.array_equal(outs2[n].numpy(), ref[n]), n
     with pytest.raises(F.FeplbError):
         case.ctx.host_wait(2)
     case.close()
