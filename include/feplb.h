@@ -325,14 +325,17 @@ int feplb_moe_forward_host(feplb_ctx* ctx, const void* x_host, const int32_t* to
                            int32_t* slot_to_row, int32_t* row_to_token, void* out_dev, void* out_host,
                            feplb_plan_out* plan_copy, void* stream);
 
-/* Pipelined form of feplb_moe_forward_host for back-to-back micro-batches.  `slot` (0 or 1) names
- * one of two caller-owned staging sets (x_dev, ids_dev, gates_dev, out_dev and the host buffers
- * must differ between the two slots; the other buffers are shared).  The call copies the inputs
+/* Pipelined form of feplb_moe_forward_host for back-to-back micro-batches.  `slot`
+ * (0 .. FEPLB_HOST_SLOTS-1) names one of the caller-owned staging sets (x_dev, ids_dev, gates_dev,
+ * out_dev and the host buffers must differ between slots in use; the other buffers are shared;
+ * two slots suffice to overlap copies with kernels, more keep the host from waiting on a result
+ * copy that is still in flight before it can launch the next forward).  The call copies the inputs
  * on the context's input stream, runs the forward on `stream` once they have arrived, copies the
  * result to out_host on the context's output stream, and returns without waiting for any of it
  * (it still blocks briefly for the planner, like feplb_moe_forward).  So the copies of micro-batch
  * i+1 overlap the kernels of micro-batch i.  Before reusing a slot's host buffers, or reading
  * out_host, call feplb_host_wait(ctx, slot). */
+#define FEPLB_HOST_SLOTS 4
 int feplb_moe_forward_host_async(feplb_ctx* ctx, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
                                  const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev,
                                  const void* w1, const void* w3, const void* w2, const uint8_t* dyn_mask_host,

@@ -54,10 +54,11 @@ struct feplb_ctx {
   void* d_preact = nullptr;   // caller-owned [s_cap, 2f]: pass 1 saves a | b there when set (training)
   // pinned staging
   int32_t* h_counts = nullptr;
-  feplb_group* h_dyn_groups = nullptr;
+  feplb_group* h_dyn_groups = nullptr;          // pinned and mapped: the upload kernel reads it through h_dyn_groups_dev
+  feplb_group* h_dyn_groups_dev = nullptr;
   uint32_t* h_status = nullptr;
   uint8_t* h_mask = nullptr;
-  int32_t* h_ready_flag = nullptr;   // pinned: sequence number of the forward whose counts are in h_counts
+  unsigned long long* h_counts_tagged = nullptr;   // pinned, written by the scan kernel: (sequence number << 32) | count
   int32_t flag_seq = 0;
   int32_t job_flag_seq = 0;          // 0: the job waits on ev_counts instead
   int32_t planner_timeout_ms = 2000; // bound of the planner's wait for the counts
@@ -65,9 +66,9 @@ struct feplb_ctx {
   cudaStream_t copy_stream = nullptr;
   // pipelined host-buffer path: input and output copy streams and per-slot events
   cudaStream_t in_stream = nullptr, out_stream = nullptr;
-  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
-  bool slot_used[2] = {false, false};
-  bool slot_staged[2] = {false, false};        // inputs already on their way (feplb_host_stage_inputs)
+  cudaEvent_t ev_in[FEPLB_HOST_SLOTS] = {}, ev_done[FEPLB_HOST_SLOTS] = {}, ev_out[FEPLB_HOST_SLOTS] = {};
+  bool slot_used[FEPLB_HOST_SLOTS] = {};
+  bool slot_staged[FEPLB_HOST_SLOTS] = {};     // inputs already on their way (feplb_host_stage_inputs)
   cudaEvent_t ev_counts = nullptr, ev_plan = nullptr;
   cudaEvent_t evr[kEvRing][EV_N] = {{nullptr}};
   cudaEvent_t* ev = evr[0];        // event set of the current forward
@@ -134,12 +135,18 @@ void planner_main(feplb_ctx* c) {
     }
     int rc = FEPLB_OK;
     // bounded wait for the counts: either the scan kernel writes them straight into pinned host
-    // memory and raises a sequence flag (whole-layer path), or a copy was enqueued and its event is
+    // memory, each tagged with the forward's sequence number (whole-layer path), or a copy was enqueued and its event is
     // polled (stand-alone feplb_plan_async); no blocking driver call either way
     const auto w0 = clk::now();
     for (uint32_t spin = 0;; ++spin) {
       if (c->job_flag_seq) {
-        if (*(volatile int32_t*)c->h_ready_flag == c->job_flag_seq) break;
+        int e = 0;
+        for (; e < c->cfg.E; ++e) {
+          const unsigned long long v = *(volatile unsigned long long*)(c->h_counts_tagged + e);
+          if ((int32_t)(v >> 32) != c->job_flag_seq) break;
+          c->h_counts[e] = (int32_t)(uint32_t)v;
+        }
+        if (e == c->cfg.E) break;
       } else {
         cudaError_t q = cudaEventQuery(c->ev_counts);
         if (q == cudaSuccess) break;
@@ -205,7 +212,7 @@ void planner_main(feplb_ctx* c) {
         for (int i = 0; i < n; ++i) dyn_rows += c->h_dyn_groups[i].rows;
         c->dyn_pair = c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (n > 0 && dyn_rows >= (int64_t)512 * n);
         cudaError_t e = cudaSuccess;
-        if (n) e = cudaMemcpyAsync(c->d_dyn_groups, c->h_dyn_groups, sizeof(feplb_group) * n, cudaMemcpyHostToDevice, c->copy_stream);
+        if (n) e = feplb_launch_upload_groups(c->h_dyn_groups_dev, c->d_dyn_groups, n, c->copy_stream);
         if (e == cudaSuccess) e = cudaEventRecord(c->ev_plan, c->copy_stream);
         if (e != cudaSuccess) rc = FEPLB_E_CUDA;
       }
@@ -272,7 +279,7 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   ok = ok && cudaMalloc(&c->d_pad_off, sizeof(int32_t) * (cfg->E + 1)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_home_groups, sizeof(feplb_group) * cfg->E) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->d_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_dyn_groups, (sizeof(feplb_group) * cap_groups + 15) / 16 * 16) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_mask, cfg->E) == cudaSuccess;
   if (cfg->phase2_copy && (int64_t)cfg->R * cfg->max_num_dyn > 30000) ok = false;   // slot ids travel in 15 bits
   if (ok && cfg->phase2_copy) {
@@ -283,16 +290,17 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
     ok = ok && cudaMalloc(&c->d_recv_w2, per * n) == cudaSuccess;
   }
   ok = ok && cudaMallocHost(&c->h_counts, sizeof(int32_t) * cfg->E) == cudaSuccess;
-  ok = ok && cudaMallocHost(&c->h_dyn_groups, sizeof(feplb_group) * cap_groups) == cudaSuccess;
+  ok = ok && cudaHostAlloc(&c->h_dyn_groups, (sizeof(feplb_group) * cap_groups + 15) / 16 * 16, cudaHostAllocMapped) == cudaSuccess &&
+       cudaHostGetDevicePointer(&c->h_dyn_groups_dev, c->h_dyn_groups, 0) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_status, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaMallocHost(&c->h_mask, cfg->E) == cudaSuccess;
-  ok = ok && cudaMallocHost(&c->h_ready_flag, sizeof(int32_t)) == cudaSuccess;
-  if (ok) *c->h_ready_flag = 0;
+  ok = ok && cudaMallocHost(&c->h_counts_tagged, sizeof(unsigned long long) * (cfg->E > 0 ? cfg->E : 1)) == cudaSuccess;
+  if (ok) memset(c->h_counts_tagged, 0, sizeof(unsigned long long) * cfg->E);
   ok = ok && cudaMemset(c->d_status, 0, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess;
-  for (int i = 0; ok && i < 2; ++i)
+  for (int i = 0; ok && i < FEPLB_HOST_SLOTS; ++i)
     ok = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming) == cudaSuccess;
@@ -345,11 +353,11 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFreeHost(c->h_dyn_groups);
   cudaFreeHost(c->h_status);
   cudaFreeHost(c->h_mask);
-  cudaFreeHost(c->h_ready_flag);
+  cudaFreeHost(c->h_counts_tagged);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->in_stream) cudaStreamDestroy(c->in_stream);
   if (c->out_stream) cudaStreamDestroy(c->out_stream);
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < FEPLB_HOST_SLOTS; ++i) {
     if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
     if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
     if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
@@ -527,6 +535,7 @@ extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out*
   }
   if (dyn_groups_dev) *dyn_groups_dev = c->d_dyn_groups;
   if (n_dyn_groups) *n_dyn_groups = c->n_dyn_groups;
+  if (c->n_dyn_groups > 0) ++c->launches;      // the planner thread's table upload kernel
   CUDA_TRY(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_plan, 0));
   return FEPLB_OK;
 }
@@ -608,7 +617,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   const int32_t seq = c->flag_seq;
   CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
                                        rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
-                                       (int64_t)c->s_cap, c->d_status, c->h_counts, c->h_ready_flag, seq, st,
+                                       (int64_t)c->s_cap, c->d_status, c->h_counts_tagged, seq, st,
                                        &c->launches));
   c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
   if ((rc = plan_kick_flag(c, dyn_mask_host, seq)) != FEPLB_OK) return rc;
@@ -680,7 +689,7 @@ extern "C" int feplb_moe_forward_host(feplb_ctx* c, const void* x_host, const in
 extern "C" int feplb_host_stage_inputs(feplb_ctx* c, int32_t slot, const void* x_host, const int32_t* topk_ids_host,
                                        const float* gates_host, void* x_dev, int32_t* ids_dev, float* gates_dev) {
   if (!c) return FEPLB_E_INVALID;
-  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "host_stage_inputs: slot must be 0 or 1");
+  if (slot < 0 || slot >= FEPLB_HOST_SLOTS) return fail(c, FEPLB_E_INVALID, "host_stage_inputs: slot out of range");
   if (c->slot_staged[slot]) return fail(c, FEPLB_E_STATE, "host_stage_inputs: slot %d already holds staged inputs", slot);
   const feplb_config& g = c->cfg;
   const size_t nx = (size_t)g.T * g.d * 2, nk = (size_t)g.T * g.K * 4;
@@ -705,7 +714,7 @@ extern "C" int feplb_moe_forward_host_async(feplb_ctx* c, int32_t slot, const vo
                                             void* y_perm, int32_t* slot_to_row, int32_t* row_to_token, void* out_dev,
                                             void* out_host, feplb_plan_out* plan_copy, void* stream) {
   if (!c) return FEPLB_E_INVALID;
-  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: slot must be 0 or 1");
+  if (slot < 0 || slot >= FEPLB_HOST_SLOTS) return fail(c, FEPLB_E_INVALID, "moe_forward_host_async: slot out of range");
   cudaStream_t st = (cudaStream_t)stream;
   const feplb_config& g = c->cfg;
   const size_t nx = (size_t)g.T * g.d * 2;
@@ -735,7 +744,7 @@ extern "C" int feplb_moe_forward_host_async(feplb_ctx* c, int32_t slot, const vo
 
 extern "C" int feplb_host_wait(feplb_ctx* c, int32_t slot) {
   if (!c) return FEPLB_E_INVALID;
-  if (slot != 0 && slot != 1) return fail(c, FEPLB_E_INVALID, "host_wait: slot must be 0 or 1");
+  if (slot < 0 || slot >= FEPLB_HOST_SLOTS) return fail(c, FEPLB_E_INVALID, "host_wait: slot out of range");
   if (c->slot_used[slot]) CUDA_TRY(c, cudaEventSynchronize(c->ev_out[slot]));
   return FEPLB_OK;
 }

@@ -45,11 +45,12 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
-                                     int32_t* counts_host, int32_t* ready_flag_host, int32_t seq,
+                                     unsigned long long* counts_host_tagged, int32_t seq,
                                      cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
                               const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,
                               cudaStream_t st, int64_t* n_launch);
+cudaError_t feplb_launch_upload_groups(const feplb_group* src_host_mapped, feplb_group* dst, int n, cudaStream_t st);
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
                                      feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row, const float* gates, void* out,

@@ -152,7 +152,7 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
              int32_t* __restrict__ rank_load_out, int32_t* __restrict__ pad_off,
              feplb_group* __restrict__ groups, uint8_t* __restrict__ mask_out,
              int32_t* __restrict__ row_to_token, int64_t s_cap,
-             int32_t* __restrict__ counts_host, volatile int32_t* ready_flag_host, int32_t seq) {
+             unsigned long long* __restrict__ counts_host_tagged, int32_t seq) {
   __shared__ int tmp[64];
   __shared__ int sc[FEPLB_MAX_EXPERTS];
   const int e = threadIdx.x;
@@ -175,10 +175,13 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
     c = run;
     counts_out[e] = c;
     sc[e] = c;
-    if (counts_host) {           // straight into pinned host memory: the planner thread polls the flag
-      counts_host[e] = c;
-      __threadfence_system();
-    }
+    // Straight into pinned host memory for the planner thread, each count in one 8-byte word that
+    // carries this forward's sequence number: the reader polls until every word shows the
+    // number, so no system-scope fence and no separate flag hold this kernel up (under bulk
+    // host<->device copies such a fence was measured to cost tens of microseconds).
+    if (counts_host_tagged)
+      *reinterpret_cast<volatile unsigned long long*>(counts_host_tagged + e) =
+          ((unsigned long long)(uint32_t)seq << 32) | (uint32_t)c;
   }
   int total;
   const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, &total);   // also orders sc[] for all threads
@@ -201,11 +204,6 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
     int sum = 0;
     for (int o = e * L; o < (e + 1) * L; ++o) sum += sc[o];
     rank_load_out[e] = sum;
-  }
-  // (the scan's barriers above ordered every thread's host writes before this flag)
-  if (counts_host && e == 0) {
-    __threadfence_system();
-    *ready_flag_host = seq;
   }
   for (int64_t i = (int64_t)total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
 }
@@ -449,6 +447,20 @@ cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const
   return launch(k_gather, blocks, kThreads, 0, st, programmatic, (const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
 }
 
+// Copies the planner's table of dynamic groups from mapped pinned host memory to the device.  A
+// kernel rather than a host-to-device memcpy: a memcpy would queue on the copy engine behind
+// whatever bulk input transfer is in flight, and the dynamic GEMM waits for this table.
+__global__ void __launch_bounds__(256) k_upload_groups(const int4* __restrict__ src_host, int4* __restrict__ dst, int n16) {
+  for (int i = threadIdx.x; i < n16; i += 256) dst[i] = src_host[i];
+}
+
+cudaError_t feplb_launch_upload_groups(const feplb_group* src_host_mapped, feplb_group* dst, int n, cudaStream_t st) {
+  const int n16 = (int)(((size_t)n * sizeof(feplb_group) + 15) / 16);      // both tables are allocated in 16-byte multiples
+  if (n16 == 0) return cudaSuccess;
+  k_upload_groups<<<1, 256, 0, st>>>(reinterpret_cast<const int4*>(src_host_mapped), reinterpret_cast<int4*>(dst), n16);
+  return cudaGetLastError();
+}
+
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
                                      feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch) {
   k_home_groups<<<1, 1024, 0, st>>>(counts, mask_in, E, E / R, A, dyn, groups, mask_out);
@@ -460,7 +472,7 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
-                                     int32_t* counts_host, int32_t* ready_flag_host, int32_t seq,
+                                     unsigned long long* counts_host_tagged, int32_t seq,
                                      cudaStream_t st, int64_t* n_launch) {
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
@@ -472,7 +484,7 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
   }
   ++*n_launch;
   return launch(k_scan_fused, 1, 1024, 0, st, true, block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off,
-                groups, mask_out, row_to_token, s_cap, counts_host, (volatile int32_t*)ready_flag_host, seq);
+                groups, mask_out, row_to_token, s_cap, counts_host_tagged, seq);
 }
 
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,

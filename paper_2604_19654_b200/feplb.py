@@ -19,6 +19,7 @@ OK, E_INVALID, E_RANGE, E_CUDA, E_NOMEM, E_TIMEOUT, E_STATE, E_DEVICE = 0, -1, -
 POLICY_LITERAL, POLICY_FIRST_FIT = 0, 1
 MASK_GIVEN, MASK_REACTIVE = 0, 1
 FFN_ALL, FFN_STATIC, FFN_DYNAMIC = 0, 1, 2
+HOST_SLOTS = 4            # staging sets of the pipelined host-buffer forward (FEPLB_HOST_SLOTS)
 
 
 class Config(C.Structure):
@@ -338,7 +339,7 @@ class Context:
 
     def moe_forward_host_async(self, slot, x_host, ids_host, gates_host, x_dev, ids_dev, gates_dev, w1, w3, w2, buf,
                                out_dev, out_host, dyn_mask_host=None, stream=None):
-        """Pipelined host-buffer forward on staging slot 0 or 1; ``host_wait(slot)`` before reading out_host."""
+        """Pipelined host-buffer forward on staging slot 0..HOST_SLOTS-1; ``host_wait(slot)`` before reading out_host."""
         mask = None if dyn_mask_host is None else np.ascontiguousarray(dyn_mask_host, np.uint8)
         self._chk(lib().feplb_moe_forward_host_async(
             self._h, int(slot), _ptr(x_host), _ptr(ids_host), _ptr(gates_host), _ptr(x_dev), _ptr(ids_dev),

@@ -432,7 +432,7 @@ def test_pipelined_host_forward_matches_the_synchronous_one():
     for n in range(len(pin)):
         assert np.array_equal(outs2[n].numpy(), ref[n]), n
     with pytest.raises(F.FeplbError):
-        case.ctx.host_wait(2)
+        case.ctx.host_wait(F.HOST_SLOTS)
     case.close()
 
 
