@@ -38,6 +38,7 @@ struct feplb_ctx {
   int64_t launches = 0;
   int gemm_pair_default = 0;   // GEMM form for launches whose group sizes the host does not know
   int gemm_pair_forced = -1;   // FEPLB_GEMM_PAIR=0/1 forces one form everywhere (experiments, tests)
+  int bwd_pair = 0;            // backward GEMMs in the pair form: bit 0 activation gradients, bit 1 weight gradients
 
   // device scratch
   int32_t* d_block_hist = nullptr;
@@ -270,6 +271,11 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   // 256-row pair tiles pay off when an expert's segment is several tiles long on average
   c->gemm_pair_default = (int64_t)cfg->T * cfg->K >= (int64_t)2048 * cfg->E;
   if (const char* e = getenv("FEPLB_GEMM_PAIR")) c->gemm_pair_default = c->gemm_pair_forced = atoi(e) != 0;
+  // backward GEMMs: the pair form pays once an expert's segment spans several 256-row tiles
+  // (measured: -7.5 % backward time at 1024 rows per expert, slower at 384); FEPLB_BWD_PAIR=0..3
+  // forces a choice (experiments, tests)
+  c->bwd_pair = (int64_t)cfg->T * cfg->K >= (int64_t)512 * cfg->E ? 3 : 0;
+  if (const char* e = getenv("FEPLB_BWD_PAIR")) c->bwd_pair = atoi(e) & 3;
   const int64_t S = (int64_t)cfg->T * cfg->K;
   c->nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   const int cap_moves = cfg->R * cfg->max_num_dyn;
@@ -881,6 +887,7 @@ extern "C" int feplb_expert_ffn_bwd(feplb_ctx* c, const void* x_perm, const void
   a.dw1 = want_w ? dw1 : nullptr; a.dw3 = dw3; a.dw2 = dw2; a.accumulate = accumulate != 0;
   a.E = c->cfg.E; a.d = c->cfg.d; a.f = c->cfg.f; a.s_cap = (int64_t)c->s_cap;
   a.status = c->d_status; a.num_sms = c->num_sms;
+  a.pair_dgrad = c->bwd_pair & 1; a.pair_wgrad = (c->bwd_pair >> 1) & 1;
   return feplb_launch_expert_ffn_bwd(a, (cudaStream_t)stream, &c->launches, c->err, sizeof(c->err));
 }
 

@@ -44,10 +44,25 @@ constexpr int kEpiStageBytes = 32 * 128;
 constexpr int kWgStages = 3;
 constexpr int kWgBufs = 4;
 static_assert(kWgBufs * kEpiWarps * kEpiStageBytes <= kABytes + kBBytesMax + kEpiWarps * kEpiStageBytes, "staging fits the freed stage");
+// Pair form (cta_group::2): a cluster of two CTAs computes a 256 x 256 tile; each CTA stages its own
+// 128 rows (columns, for the MN-major kind) of A and half of the B tile, 32 KiB per stage.
+constexpr int kPairStageBytes = kABytes + 128 * BK * 2;
+constexpr int kPairStages = 6;
+constexpr int kPairWgStages = 4;
+constexpr int kMaxStages = 6;
+
+template <int KIND, bool PAIR>
+struct Ring {
+  static constexpr int kNS = PAIR ? (KIND == 2 ? kPairWgStages : kPairStages) : (KIND == 2 ? kWgStages : kStages);
+  static constexpr int kBytes = PAIR ? kPairStageBytes : kStageBytes;
+  static constexpr int kTileRows = PAIR ? 2 * BM : BM;
+  static_assert(kNS <= kMaxStages && kNS * kBytes + (KIND == 2 ? kWgBufs : 1) * kEpiWarps * kEpiStageBytes <=
+                kStages * kStageBytes + kEpiWarps * kEpiStageBytes, "ring + staging fit below the tail");
+};
 
 struct Tail {
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kAccStages];
   unsigned long long tmem_empty[kAccStages];
   uint32_t tmem_base;
@@ -85,7 +100,7 @@ struct BwdParams {
 
 struct Coord { int row0, rows_valid, expert, mt, nt, kblocks; };
 
-template <int KIND>
+template <int KIND, int TR>
 __device__ __forceinline__ Coord tile_coord(const Tail* t, const BwdParams& p, int tile) {
   Coord c;
   if (KIND == KIND_WG) {
@@ -107,8 +122,8 @@ __device__ __forceinline__ Coord tile_coord(const Tail* t, const BwdParams& p, i
     if (t->prefix[mid] <= mt) lo = mid; else hi = mid;
   }
   const int local = mt - t->prefix[lo];
-  c.row0 = t->g_row_start[lo] + local * BM;
-  c.rows_valid = min(BM, t->g_rows[lo] - local * BM);
+  c.row0 = t->g_row_start[lo] + local * TR;
+  c.rows_valid = min(TR, t->g_rows[lo] - local * TR);
   c.expert = t->g_expert[lo];
   c.mt = mt;
   c.nt = tile - mt * p.n_tiles_n;
@@ -161,6 +176,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, 
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+// The same, in the pair form: the byte count is credited to an mbarrier of the pair's leader.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 // TMA store / reduce-add of one staged 32 x 32 fp32 box to dW[e] (tensor map over [E, M, N]).
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
@@ -175,14 +197,20 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-template <int KIND>
+template <int KIND, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_out, const BwdParams p) {
-  constexpr int NS = KIND == KIND_WG ? kWgStages : kStages;      // ring stages
+  constexpr int NS = Ring<KIND, PAIR>::kNS;                       // ring stages
+  constexpr int kSB = Ring<KIND, PAIR>::kBytes;                   // bytes per stage
+  constexpr int TR = Ring<KIND, PAIR>::kTileRows;                 // rows (WG: M columns) of a tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* epi_smem = smem + (size_t)NS * kStageBytes;
+  uint8_t* epi_smem = smem + (size_t)NS * kSB;
+  // pair form: rank in the cluster of two (0 = leader, issues the MMAs); tiles are dealt per cluster
+  const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   Tail* tail = reinterpret_cast<Tail*>(smem + (size_t)kStages * kStageBytes + (size_t)kEpiWarps * kEpiStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &tail->abort_flag;
@@ -198,15 +226,20 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(smem_u32(&tail->tmem_full[a]), 1);
-      mbar_init(smem_u32(&tail->tmem_empty[a]), kEpiWarps);
+      mbar_init(smem_u32(&tail->tmem_empty[a]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
     tail->abort_flag = 0;
     fence_barrier_init();
   }
   if (warp == 1) {
     __syncwarp();
-    tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(smem_u32(&tail->tmem_base), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tail->tmem_base), kTmemCols);
+      tmem_relinquish();
+    }
   }
   for (int g = threadIdx.x; g < p.n_groups; g += kThreads) {
     const feplb_group gr = p.groups[g];
@@ -214,7 +247,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int tiles = 0, rows = 0;
     if (selected && gr.rows > 0) {
       const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 && (int64_t)gr.row_start + gr.rows <= p.s_cap;
-      if (ok) { tiles = (gr.rows + BM - 1) / BM; rows = gr.rows; }
+      if (ok) { tiles = (gr.rows + TR - 1) / TR; rows = gr.rows; }
       else atomicOr(p.status, FEPLB_ST_GROUP);
     }
     tail->prefix[g + 1] = tiles;
@@ -244,11 +277,12 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (lane == 0) tail->prefix[0] = 0;
   }
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tail->tmem_base;
   const int total_tiles = KIND == KIND_WG ? p.n_groups * p.m_tiles * p.n_tiles_n : tail->prefix[p.n_groups] * p.n_tiles_n;
   const uint32_t b_half_bytes = (uint32_t)p.bn * BK * 2;
-  const uint32_t stage_tx = kABytes + 2 * b_half_bytes;
+  const uint32_t stage_tx = PAIR ? 2 * (kABytes + b_half_bytes) : kABytes + 2 * b_half_bytes;
 
   if (warp == 0) {
     // ---- TMA producer ---------------------------------------------------------------------
@@ -256,20 +290,39 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Coord c = tile_coord<KIND>(tail, p, tile);
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+        const Coord c = tile_coord<KIND, TR>(tail, p, tile);
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!(ok = mbar_wait(smem_u32(&tail->empty[stage]), phase ^ 1u, abort_flag, p.status))) break;
           const uint32_t full = smem_u32(&tail->full[stage]);
-          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kSB);
           const uint32_t sb = sa + kABytes;
+          if (PAIR) {
+            // both CTAs credit the LEADER's barrier; the leader announces the bytes of both.  Each
+            // CTA brings its own 128 rows (WG: columns) of A and its half of the B tile.
+            const uint32_t full0 = map_to_cta(full, 0);
+            if (cta_rank == 0) mbar_expect_tx(full, stage_tx);
+            if (KIND == KIND_WG) {
+              const int k0 = c.row0 + kb * BK;
+              tma_load_3d_pair(sa, &tm_a, full0, 0, k0, c.mt * (TR / 64) + (int)cta_rank * (BM / 64));
+              tma_load_3d_pair(sb, &tm_b0, full0, 0, k0, c.nt * (2 * p.bn / 64) + (int)cta_rank * (p.bn / 64));
+            } else {
+              const CUtensorMap* mb = (KIND == KIND_DX && kb >= p.k_switch) ? &tm_b1 : &tm_b0;
+              const int kb_b = (KIND == KIND_DX && kb >= p.k_switch) ? kb - p.k_switch : kb;
+              const int brow = c.expert * p.b_rows_per_expert + c.nt * 2 * p.bn + (int)cta_rank * p.bn;
+              tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
+              tma_load_2d_pair(sb, mb, full0, kb_b * BK, brow);
+            }
+            if (++stage == NS) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           mbar_expect_tx(full, stage_tx);
           if (KIND == KIND_WG) {
             // K runs along the expert's rows: both operands are read as they lie in memory (row = K,
             // columns = M resp. N contiguous).  The maps see a matrix as [64-column chunk][row][64
             // columns], so one load brings 64 rows of all the tile's chunks, 8 KiB per chunk.
             const int k0 = c.row0 + kb * BK;
-            tma_load_3d(sa, &tm_a, full, 0, k0, c.mt * (BM / 64));
+            tma_load_3d(sa, &tm_a, full, 0, k0, c.mt * (TR / 64));
             tma_load_3d(sb, &tm_b0, full, 0, k0, c.nt * (2 * p.bn / 64));
           } else {
             const CUtensorMap* mb = (KIND == KIND_DX && kb >= p.k_switch) ? &tm_b1 : &tm_b0;
@@ -288,39 +341,41 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
   } else if (warp == 1) {
     // ---- MMA issuer -------------------------------------------------------------------------
-    if (lane == 0) {
-      const uint32_t idesc = KIND == KIND_WG ? make_idesc_mn(BM, 2 * p.bn) : make_idesc(BM, 2 * p.bn);
+    if (lane == 0 && cta_rank == 0) {
+      const uint32_t idesc = KIND == KIND_WG ? make_idesc_mn(TR, 2 * p.bn) : make_idesc(TR, 2 * p.bn);
       int stage = 0, as = 0;
       uint32_t phase = 0, aphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const Coord c = tile_coord<KIND>(tail, p, tile);
+      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+        const Coord c = tile_coord<KIND, TR>(tail, p, tile);
         if (!(ok = mbar_wait(smem_u32(&tail->tmem_empty[as]), aphase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * kAccCols);
         for (int kb = 0; kb < c.kblocks; ++kb) {
           if (!(ok = mbar_wait(smem_u32(&tail->full[stage]), phase, abort_flag, p.status))) break;
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
-          if (KIND == KIND_WG) {
-            const uint64_t da = make_smem_desc_mn(sa);
-            const uint64_t db = make_smem_desc_mn(sa + kABytes);
+          const uint32_t sa = smem_u32(smem + (size_t)stage * kSB);
+          // descriptor step per UMMA_K: MN-major 16 K rows of 128 bytes (2048 >> 4), K-major 32 bytes (>> 4)
+          const uint64_t da = KIND == KIND_WG ? make_smem_desc_mn(sa) : make_smem_desc(sa);
+          const uint64_t db = KIND == KIND_WG ? make_smem_desc_mn(sa + kABytes) : make_smem_desc(sa + kABytes);
+          constexpr uint64_t kStep = KIND == KIND_WG ? 128 : 2;
 #pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)    // 16 K rows of 128 bytes per step
-              umma_bf16(d_tmem, da + (uint64_t)(k * 128), db + (uint64_t)(k * 128), idesc, (uint32_t)((kb | k) != 0));
-          } else {
-            const uint64_t da = make_smem_desc(sa);
-            const uint64_t db = make_smem_desc(sa + kABytes);
-#pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)
-              umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (uint32_t)((kb | k) != 0));
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            if (PAIR) umma_bf16_pair(d_tmem, da + kStep * k, db + kStep * k, idesc, (uint32_t)((kb | k) != 0));
+            else umma_bf16(d_tmem, da + kStep * k, db + kStep * k, idesc, (uint32_t)((kb | k) != 0));
           }
-          umma_commit(smem_u32(&tail->empty[stage]));
+          if (PAIR) umma_commit_pair(smem_u32(&tail->empty[stage]));
+          else umma_commit(smem_u32(&tail->empty[stage]));
           if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        if (c.kblocks > 0) umma_commit(smem_u32(&tail->tmem_full[as]));
-        else mbar_arrive(smem_u32(&tail->tmem_full[as]));     // an expert without rows: nothing was issued
+        if (c.kblocks > 0) {
+          if (PAIR) umma_commit_pair(smem_u32(&tail->tmem_full[as]));
+          else umma_commit(smem_u32(&tail->tmem_full[as]));
+        } else {                                                 // an expert without rows: nothing was issued
+          mbar_arrive(smem_u32(&tail->tmem_full[as]));
+          if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tail->tmem_full[as]), 1));
+        }
         if (++as == kAccStages) { as = 0; aphase ^= 1u; }
       }
     }
@@ -332,8 +387,8 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int as = 0;
     uint32_t aphase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-      const Coord c = tile_coord<KIND>(tail, p, tile);
+    for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+      const Coord c = tile_coord<KIND, TR>(tail, p, tile);
       ok = mbar_wait(smem_u32(&tail->tmem_full[as]), aphase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -344,7 +399,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // fp32 tile of dW[e]: this warp's 32 rows, 32 columns at a time: TMEM -> registers ->
         // swizzled staging buffer -> one TMA store (or reduce-add into dW) of the 32 x 32 box.
         // An expert without rows adds nothing; without accumulation it gets zeros.
-        const int m0 = c.mt * BM + q * 32;
+        const int m0 = c.mt * TR + (int)cta_rank * BM + q * 32;
         const bool emit = m0 < p.m_total && !(c.kblocks == 0 && p.accumulate);
         for (int col = 0; col < out_cols; col += 32) {
           const int n0 = c.nt * out_cols + col;
@@ -376,7 +431,7 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (++wg_buf == kWgBufs) wg_buf = 0;
         }
       } else {
-        const int row_off = q * 32;
+        const int row_off = (int)cta_rank * BM + q * 32;
         const int rows_here = c.rows_valid - row_off;
         const int my_row = c.row0 + row_off + lane;
         const bool row_ok = lane < rows_here;
@@ -431,7 +486,10 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tail->tmem_empty[as]), 0));
+        else mbar_arrive(smem_u32(&tail->tmem_empty[as]));
+      }
       if (++as == kAccStages) { as = 0; aphase ^= 1u; }
     }
     if (KIND == KIND_WG && lane == 0) bulk_wait_read<0>();      // staging must outlive the stores that read it
@@ -439,10 +497,12 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory: leave together
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -591,17 +651,41 @@ bool make_tmap_out(CUtensorMap* m, float* base, uint64_t E, uint64_t M, uint64_t
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int KIND>
+template <int KIND, bool PAIR>
 cudaError_t launch_kind(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tout,
-                        const BwdParams& p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_ffn_bwd_gemm<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
+                        const BwdParams& p, int num_sms, cudaStream_t st) {
+  static int grid = 0;   // per instantiation: set on first use
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  cfg.attrs = at;
+  cfg.numAttrs = 0;
+  if (PAIR) {
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.numAttrs = 1;
   }
-  k_ffn_bwd_gemm<KIND><<<grid, kThreads, kSmemBytes, st>>>(ta, tb0, tb1, tout, p);
-  return cudaGetLastError();
+  if (!grid) {
+    cudaError_t e = cudaFuncSetAttribute(k_ffn_bwd_gemm<KIND, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    int g = num_sms;
+    if (PAIR) {
+      // as many clusters of two as can be resident at once (one CTA per SM, both SMs in one GPC)
+      int n_clusters = 0;
+      cfg.gridDim = dim3(num_sms / 2 * 2);
+      e = cudaOccupancyMaxActiveClusters(&n_clusters, k_ffn_bwd_gemm<KIND, PAIR>, &cfg);
+      if (e != cudaSuccess) return e;
+      if (n_clusters < 1) return cudaErrorLaunchOutOfResources;
+      g = 2 * (n_clusters < num_sms / 2 ? n_clusters : num_sms / 2);
+    }
+    grid = g;
+  }
+  cfg.gridDim = dim3(grid);
+  return cudaLaunchKernelEx(&cfg, k_ffn_bwd_gemm<KIND, PAIR>, ta, tb0, tb1, tout, p);
 }
 
 cudaError_t transpose(const void* src, void* dst, int rows, int cols, int64_t ld_src, int64_t ld_dst, int batch,
@@ -664,14 +748,16 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
   BwdParams ph = p;
   ph.n_tiles_n = (f + 2 * bn_h - 1) / (2 * bn_h); ph.n_limit = f; ph.num_k_blocks = d / BK; ph.b_rows_per_expert = f; ph.bn = bn_h;
   ph.out = (__nv_bfloat16*)a.d_ab; ph.ld_out = 2 * f; ph.ab = (const __nv_bfloat16*)a.ab_saved; ph.f = f;
-  e = launch_kind<KIND_DH>(tm_dy, tm_w2t, tm_w2t, tm_dy, ph, a.num_sms, st);
+  e = a.pair_dgrad ? launch_kind<KIND_DH, true>(tm_dy, tm_w2t, tm_w2t, tm_dy, ph, a.num_sms, st)
+                   : launch_kind<KIND_DH, false>(tm_dy, tm_w2t, tm_w2t, tm_dy, ph, a.num_sms, st);
   ++*n_launch;
   if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DH>");
   // ---- dX = [dA | dB] [W1^T ; W3^T] ------------------------------------------------------------------
   BwdParams px = p;
   px.n_tiles_n = d / (2 * bn_x); px.n_limit = d; px.num_k_blocks = 2 * f / BK; px.k_switch = f / BK; px.b_rows_per_expert = d; px.bn = bn_x;
   px.out = (__nv_bfloat16*)a.d_x_perm; px.ld_out = d;
-  e = launch_kind<KIND_DX>(tm_dab, tm_w1t, tm_w3t, tm_dab, px, a.num_sms, st);
+  e = a.pair_dgrad ? launch_kind<KIND_DX, true>(tm_dab, tm_w1t, tm_w3t, tm_dab, px, a.num_sms, st)
+                   : launch_kind<KIND_DX, false>(tm_dab, tm_w1t, tm_w3t, tm_dab, px, a.num_sms, st);
   ++*n_launch;
   if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<DX>");
   if (!a.dw1) return FEPLB_OK;
@@ -695,16 +781,17 @@ int feplb_launch_expert_ffn_bwd(const feplb_bwd_args& a, cudaStream_t st, int64_
     const int bn = (j.n_total % 256 == 0) ? 128 : 64;
     CUtensorMap tm_at, tm_bt, tm_o;
     if (!make_tmap_mn(&tm_at, j.p, (uint64_t)a.s_cap, (uint64_t)j.m_total, (uint64_t)j.ld_p, BM / 64) ||
-        !make_tmap_mn(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, 2 * bn / 64) ||
+        !make_tmap_mn(&tm_bt, j.q, (uint64_t)a.s_cap, (uint64_t)j.n_total, (uint64_t)j.n_total, (a.pair_wgrad ? bn : 2 * bn) / 64) ||
         !make_tmap_out(&tm_o, j.out, (uint64_t)a.E, (uint64_t)j.m_total, (uint64_t)j.n_total)) {
       snprintf(err, errn, "cuTensorMapEncodeTiled failed (weight gradient)");
       return FEPLB_E_CUDA;
     }
     BwdParams pw = p;
     pw.groups = a.expert_table; pw.n_groups = a.E; pw.which = FEPLB_FFN_ALL;
-    pw.bn = bn; pw.n_tiles_n = (j.n_total + 2 * bn - 1) / (2 * bn); pw.m_tiles = (j.m_total + BM - 1) / BM;
+    pw.bn = bn; pw.n_tiles_n = (j.n_total + 2 * bn - 1) / (2 * bn); pw.m_tiles = a.pair_wgrad ? (j.m_total + 2 * BM - 1) / (2 * BM) : (j.m_total + BM - 1) / BM;
     pw.m_total = j.m_total; pw.n_total = j.n_total; pw.wout = j.out; pw.accumulate = a.accumulate;
-    e = launch_kind<KIND_WG>(tm_at, tm_bt, tm_bt, tm_o, pw, a.num_sms, st);
+    e = a.pair_wgrad ? launch_kind<KIND_WG, true>(tm_at, tm_bt, tm_bt, tm_o, pw, a.num_sms, st)
+                     : launch_kind<KIND_WG, false>(tm_at, tm_bt, tm_bt, tm_o, pw, a.num_sms, st);
     ++*n_launch;
     if (e != cudaSuccess) return fail_cuda("k_ffn_bwd_gemm<WG>");
   }

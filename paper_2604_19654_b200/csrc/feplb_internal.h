@@ -85,6 +85,7 @@ struct feplb_bwd_args {
   float* dw1; float* dw3; float* dw2; int accumulate;       // fp32 [E,f,d], [E,f,d], [E,d,f]; dw1 == nullptr: skip
   int E, d, f; int64_t s_cap;
   uint32_t* status; int num_sms;
+  int pair_dgrad, pair_wgrad;                               // 1: cta_group::2 form (256 x 256 tiles per cluster of two CTAs)
 };
 cudaError_t feplb_launch_transpose_weights(const void* w1, const void* w3, const void* w2, void* w1t, void* w3t, void* w2t,
                                            int E, int d, int f, cudaStream_t st, int64_t* n_launch);

@@ -63,9 +63,13 @@ def _run_backward(w, mb=0, scale=1.0, **cfg_kw):
     return case, bwd, (dw1, dw3, dw2), ref, (w1t, w3t, w2t), d_out
 
 
+@pytest.mark.parametrize("pair", [0, 3])
 @pytest.mark.parametrize("name,T", [("cfg1", 256), ("cfg2", 384), ("cfg4", 512)])
-def test_backward_parity(name, T):
+def test_backward_parity(name, T, pair, monkeypatch):
+    """``pair``: both forms of the backward GEMMs (single CTA per 128-row tile; clusters of two CTAs on
+    256-row tiles), forced through the environment switch the context reads when it is created."""
     import torch
+    monkeypatch.setenv("FEPLB_BWD_PAIR", str(pair))
     w = W.get_workload(name).with_(T=T)
     if name != "cfg1":
         w = w.with_(E=16, R=4)                       # fewer experts: the fp64 reference stays cheap
