@@ -401,17 +401,10 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // An expert without rows adds nothing; without accumulation it gets zeros.
         const int m0 = c.mt * TR + (int)cta_rank * BM + q * 32;
         const bool emit = m0 < p.m_total && !(c.kblocks == 0 && p.accumulate);
-        for (int col = 0; col < out_cols; col += 32) {
+        // one 32-column chunk: registers -> staging buffer -> TMA store / reduce-add
+        auto put = [&](const uint32_t (&a)[32], int col) {
           const int n0 = c.nt * out_cols + col;
-          if (!emit || n0 >= p.n_total) continue;     // warp-uniform; M and N are multiples of 32
-          uint32_t a[32];
-          if (c.kblocks > 0) {
-            tmem_ld32(taddr + (uint32_t)col, a);
-            tmem_ld_wait();
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) a[i] = 0u;
-          }
+          if (n0 >= p.n_total) return;                        // warp-uniform; M and N are multiples of 32
           const uint32_t buf = stg + (uint32_t)(wg_buf * kEpiStageBytes);
           if (lane == 0) bulk_wait_read<kWgBufs - 1>();     // the store that read this buffer kWgBufs boxes ago
           __syncwarp();
@@ -429,6 +422,25 @@ k_ffn_bwd_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             bulk_commit();
           }
           if (++wg_buf == kWgBufs) wg_buf = 0;
+        };
+        if (emit) {
+          uint32_t a0[32], a1[32];
+          if (c.kblocks > 0) {
+            // the TMEM load of the next chunk is in flight while the current one is staged and sent
+            tmem_ld32(taddr, a0);
+            for (int col = 0; col < out_cols; col += 64) {
+              tmem_ld_wait();
+              tmem_ld32(taddr + (uint32_t)(col + 32), a1);
+              put(a0, col);
+              tmem_ld_wait();
+              if (col + 64 < out_cols) tmem_ld32(taddr + (uint32_t)(col + 64), a0);
+              put(a1, col + 32);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) a0[i] = 0u;
+            for (int col = 0; col < out_cols; col += 32) put(a0, col);
+          }
         }
       } else {
         const int row_off = (int)cta_rank * BM + q * 32;
