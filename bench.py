@@ -162,6 +162,8 @@ def _config_dict(w, args, extra=None):
          "routing": f"{w.routing}(alpha={w.alpha})", "parallelism": f"dp{args.gpus} (independent micro-batches per rank)",
          "cache": "inputs rotate over the micro-batches; weights (%.2f GiB) exceed the 126 MB L2"
                   % (3 * w.E * w.d * w.f * 2 / 2 ** 30)}
+    if getattr(args, "split", False):
+        c["plan"] = "split extension on (not in the paper)"
     if extra:
         c.update(extra)
     return c
@@ -211,7 +213,7 @@ def run_cuda(args, w):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.build()
-    cfg = F.config_from_workload(w, phase2_copy=1 if args.phase2 else 0)
+    cfg = F.config_from_workload(w, phase2_copy=1 if args.phase2 else 0, split=1 if args.split else 0)
     ctx = F.Context(cfg)
     buf = F.Buffers(cfg)
 
@@ -491,11 +493,12 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
         roof = {"bound": "tensor", "kernel": "k_grouped_gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak if achieved else None, "peak_source": peaks["source"] + " (sustained)",
                 "frac_of_burst": achieved / peaks["bf16_tflops"] if achieved else None,
+                "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
                 "launches_timed": gemm_launches, "avg_launch_us": ffn_us / gemm_launches if gemm_launches else None,
                 "dispatch_gbs": io_bytes / (totals["dev_dispatch_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_dispatch_us"] else None,
                 "combine_gbs": io_bytes / (totals["dev_combine_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_combine_us"] else None,
-                "hbm_peak_gbs": peaks["hbm_gbs"]}
+                "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_nominal_gbs": 7700.0}
         stage_us = {k: (v / n_fw if n_fw else None) for k, v in totals.items()}
         # CPU oracle on the host cores: a bounded sample of the same workload
         cpu = None
@@ -530,7 +533,7 @@ def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb,
     """Token straggler from the plans and GEMM straggler from per-virtual-rank launches, before
     (every group on its home rank) and after rebalancing, averaged over the micro-batches."""
     import torch
-    tok_b, tok_a, gem_b, gem_a, gem_bm, gem_am = [], [], [], [], [], []
+    tok_b, tok_a, gem_b, gem_a, gem_bm, gem_am, tok_bm, tok_am = [], [], [], [], [], [], [], []
     L = w.E // w.R
     for i in range(min(n_mb, 4)):
         x, ids, g = dev[i]
@@ -539,6 +542,8 @@ def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb,
         lb, la = p.load_before.astype(np.float64), p.load_after.astype(np.float64)
         tok_b.append(lb.max() / lb.mean())
         tok_a.append(la.max() / la.mean())
+        tok_bm.append(lb.max() - lb.mean())
+        tok_am.append(la.max() - la.mean())
         groups = p.groups
         per_rank = {"before": [], "after": []}
         for label, key in (("before", lambda gr: gr[0] // L), ("after", lambda gr: gr[3])):
@@ -562,7 +567,12 @@ def measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb,
         gem_a.append(a.max() / a.mean())
         gem_bm.append(b.max() - b.mean())
         gem_am.append(a.max() - a.mean())
+    def min_gain(before, after):      # smallest per-micro-batch reduction of max - mean (1 = all of it removed)
+        return float(min(1.0 - a / b if b > 0 else 0.0 for b, a in zip(before, after)))
     return {"token_ratio_before": float(np.mean(tok_b)), "token_ratio_after": float(np.mean(tok_a)),
+            "token_max_minus_mean_rows_before": float(np.mean(tok_bm)), "token_max_minus_mean_rows_after": float(np.mean(tok_am)),
+            "token_min_gain_over_micro_batches": min_gain(tok_bm, tok_am),
+            "gemm_min_gain_over_micro_batches": min_gain(gem_bm, gem_am),
             "gemm_ratio_before": float(np.mean(gem_b)), "gemm_ratio_after": float(np.mean(gem_a)),
             "gemm_max_minus_mean_ms_before": float(np.mean(gem_bm)), "gemm_max_minus_mean_ms_after": float(np.mean(gem_am)),
             "micro_batches": len(tok_b), "definition": "max over virtual ranks / mean; GEMM time = expert FFN of one rank's groups run alone"}
@@ -577,6 +587,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-sample-tokens", type=int, default=1024)
     ap.add_argument("--no-straggler", action="store_true")
+    ap.add_argument("--split", action="store_true",
+                    help="plan with the splitting extension (a hot expert is cut in multiples of the granule; not in the paper)")
     ap.add_argument("--backward", action="store_true", help="also time forward + backward (weight gradients included)")
     ap.add_argument("--phase2", action="store_true",
                     help="really copy migrated experts' weights into the receive buffer (copy engines) during the static GEMM")

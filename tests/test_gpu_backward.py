@@ -96,6 +96,29 @@ def test_backward_parity(name, T, pair, monkeypatch):
     case.close()
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_backward_random_shapes(seed, monkeypatch):
+    """Seeded random small layers (odd token counts, 1-4 ranks, ragged tiles, experts without rows),
+    both GEMM forms."""
+    rng = np.random.default_rng(9100 + seed)
+    R = int(rng.choice([1, 2, 4]))
+    L = int(rng.choice([1, 2, 3, 6]))
+    E = R * L
+    w = W.get_workload("cfg2").with_(
+        name=f"randb{seed}", T=int(rng.integers(1, 500)), E=E, R=R, K=int(rng.integers(1, min(E, 6) + 1)),
+        d=int(rng.choice([128, 256, 384])), f=int(rng.choice([64, 192, 256])), dyn=int(rng.integers(0, L + 1)),
+        max_num_dyn=2, tau=8, routing="dirichlet", alpha=float(rng.choice([0.1, 0.5])))
+    monkeypatch.setenv("FEPLB_BWD_PAIR", str(int(rng.choice([0, 3]))))
+    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w, mb=seed)
+    rdx, rdg, rdw1, rdw3, rdw2 = ref
+    _close(W.bf16_bits_to_f64(F.bf16_bits(bwd.d_x))[: w.T], rdx, "dx")
+    _close(bwd.d_gates.cpu().numpy().astype(np.float64)[: w.T], rdg, "dgates")
+    _close(dw2.cpu().numpy().astype(np.float64), rdw2, "dw2")
+    _close(dw1.cpu().numpy().astype(np.float64), rdw1, "dw1")
+    _close(dw3.cpu().numpy().astype(np.float64), rdw3, "dw3")
+    case.close()
+
+
 def test_combine_bwd_bit_exact_rows_and_gate_gradients():
     import torch
     w = W.get_workload("cfg2").with_(T=300, E=16, R=4)

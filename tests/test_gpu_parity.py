@@ -287,6 +287,31 @@ def test_forward_cfg1(A):
     case.close()
 
 
+def _random_workload(seed):
+    """A seeded random small layer: odd token counts, expert counts that are not powers of two,
+    several ranks, widths that give two to six 64-wide K blocks and ragged N tiles."""
+    rng = np.random.default_rng(4200 + seed)
+    R = int(rng.choice([1, 2, 3, 4]))
+    L = int(rng.choice([1, 2, 3, 5, 8]))
+    E = R * L
+    K = int(rng.integers(1, min(E, 8) + 1))
+    w = W.get_workload("cfg2").with_(
+        name=f"rand{seed}", T=int(rng.integers(1, 700)), E=E, R=R, K=K,
+        d=int(rng.choice([128, 256, 384])), f=int(rng.choice([64, 128, 192, 256])),
+        dyn=int(rng.integers(0, L + 1)), max_num_dyn=int(rng.integers(0, 4)), tau=int(rng.choice([0, 1, 8, 64])),
+        routing=str(rng.choice(["dirichlet", "zipf"])), alpha=float(rng.choice([0.2, 0.5, 1.2])))
+    return w, int(rng.choice([1, 128])), int(rng.integers(0, 2)), int(rng.integers(0, 2))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_forward_random_shapes(seed, monkeypatch):
+    w, A, split, pair = _random_workload(seed)
+    monkeypatch.setenv("FEPLB_GEMM_PAIR", str(pair))
+    case = DeviceCase(w, mb=seed, row_align=A, split=split, split_granule=128 if A == 128 else 16)
+    _check_forward(case)
+    case.close()
+
+
 @pytest.mark.parametrize("seed", range(4))
 def test_forward_cfg1_other_seeds(seed):
     w = W.get_workload("cfg1")
