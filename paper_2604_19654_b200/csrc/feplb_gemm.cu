@@ -458,7 +458,11 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
 template <bool SWIGLU, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tr0,
                        const CUtensorMap& tr1, const GemmParams& p, int num_sms, cudaStream_t st) {
-  static int grid = 0;   // per instantiation: set on first use
+  // per instantiation and device: the shared-memory attribute and the resident grid are set on first use
+  static int grid_of[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  int& grid = grid_of[dev];
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;

@@ -666,7 +666,11 @@ bool make_tmap_out(CUtensorMap* m, float* base, uint64_t E, uint64_t M, uint64_t
 template <int KIND, bool PAIR>
 cudaError_t launch_kind(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tout,
                         const BwdParams& p, int num_sms, cudaStream_t st) {
-  static int grid = 0;   // per instantiation: set on first use
+  // per instantiation and device: the shared-memory attribute and the resident grid are set on first use
+  static int grid_of[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  int& grid = grid_of[dev];
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
