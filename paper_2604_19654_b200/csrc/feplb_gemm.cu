@@ -131,9 +131,39 @@ __device__ __forceinline__ void convert_slice(const uint32_t (&a)[32], const uin
 // 32 rows x 64 bf16 columns, one row per lane in packed[32]: through the warp's staging area (row
 // `lane`, 16-byte chunk j at position j ^ (lane & 7)) and out again 4 rows per instruction, so
 // that every global store covers whole 128-byte lines; rows >= rows_here are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+// The warp's staging area may still be read by the TMA store of its previous slice.
+__device__ __forceinline__ void staging_ready(int lane) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  __syncwarp();
+}
+
+// Full slices (all 32 rows valid) leave through one TMA store: the staging layout below IS the
+// 128-byte-swizzled box layout, so lane 0 hands the 4 KiB to the copy unit and the warp moves on.
+__device__ __forceinline__ void stage_and_tma_store(uint32_t stg, const uint32_t* packed, const CUtensorMap* m, int gcol,
+                                                    int grow, int lane) {
+  staging_ready(lane);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(packed[4 * j]), "r"(packed[4 * j + 1]),
+                 "r"(packed[4 * j + 2]), "r"(packed[4 * j + 3]) : "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) {
+    tma_store_2d(m, stg, gcol, grow);
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+}
+
 __device__ __forceinline__ void stage_and_store(uint32_t stg, const uint32_t* packed, __nv_bfloat16* obase, int ld,
                                                 int col, int rows_here, int lane) {
   const int rd_row = lane >> 3, rd_chunk = lane & 7;
+  staging_ready(lane);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const uint32_t addr = stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4));
@@ -156,7 +186,7 @@ template <bool SWIGLU, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_r0,
-               const __grid_constant__ CUtensorMap tm_r1, const GemmParams p) {
+               const __grid_constant__ CUtensorMap tm_r1, const __grid_constant__ CUtensorMap tm_out, const GemmParams p) {
   constexpr int kStages = Ring<PAIR>::kStages, kStageBytes = Ring<PAIR>::kStageBytes;
   constexpr int kTileRows = Ring<PAIR>::kTileRows;
   extern __shared__ uint8_t smem_raw[];
@@ -182,6 +212,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     prefetch_tmap(&tm_b1);
     prefetch_tmap(&tm_r0);
     prefetch_tmap(&tm_r1);
+    prefetch_tmap(&tm_out);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&tail->full[s]), 1);
       mbar_init(smem_u32(&tail->empty[s]), 1);
@@ -386,7 +417,8 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             tmem_ld32(taddr + (uint32_t)(p.bn + col + 96), b1);
           }
         }
-        stage_and_store(stg, packed, obase, p.ld_out, col, rows_here, lane);
+        if (rows_here >= 32) stage_and_tma_store(stg, packed, &tm_out, c.nt * out_cols + col, c.row0 + row_off, lane);
+        else stage_and_store(stg, packed, obase, p.ld_out, col, rows_here, lane);
       }
       tc_fence_before();
       __syncwarp();
@@ -396,6 +428,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       }
       if (++as == kAccStages) { as = 0; aphase ^= 1u; }
     }
+    staging_ready(lane);      // the staging area must outlive the last TMA store that reads it
   }
 
   // ---- teardown ---------------------------------------------------------------------------------
@@ -457,7 +490,7 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
 
 template <bool SWIGLU, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tr0,
-                       const CUtensorMap& tr1, const GemmParams& p, int num_sms, cudaStream_t st) {
+                       const CUtensorMap& tr1, const CUtensorMap& tout, const GemmParams& p, int num_sms, cudaStream_t st) {
   // per instantiation and device: the shared-memory attribute and the resident grid are set on first use
   static int grid_of[64] = {};
   int dev = 0;
@@ -496,7 +529,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUte
     grid = g;
   }
   cfg.gridDim = dim3(grid);
-  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, tr0, tr1, p);
+  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, tr0, tr1, tout, p);
 }
 
 }  // namespace
@@ -507,12 +540,14 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   const int bn1 = (a.f % 128 == 0) ? 128 : 64;
   // pass 2: Y = H W2;  N tile = 2*bn columns of Y
   const int bn2 = (a.d % 256 == 0) ? 128 : 64;
-  CUtensorMap tm_x, tm_w1, tm_w3, tm_h, tm_w2;
+  CUtensorMap tm_x, tm_w1, tm_w3, tm_h, tm_w2, tm_ho, tm_yo;     // tm_ho, tm_yo: outputs in boxes of 32 rows x 64 columns
   if (!make_tmap(&tm_x, a.x_perm, (uint64_t)a.s_cap, (uint64_t)a.d, BM) ||
       !make_tmap(&tm_w1, a.w1, (uint64_t)a.E * a.f, (uint64_t)a.d, bn1) ||
       !make_tmap(&tm_w3, a.w3, (uint64_t)a.E * a.f, (uint64_t)a.d, bn1) ||
       !make_tmap(&tm_h, a.h, (uint64_t)a.s_cap, (uint64_t)a.f, BM) ||
-      !make_tmap(&tm_w2, a.w2, (uint64_t)a.E * a.d, (uint64_t)a.f, bn2)) {
+      !make_tmap(&tm_w2, a.w2, (uint64_t)a.E * a.d, (uint64_t)a.f, bn2) ||
+      !make_tmap(&tm_ho, a.h, (uint64_t)a.s_cap, (uint64_t)a.f, 32) ||
+      !make_tmap(&tm_yo, a.y, (uint64_t)a.s_cap, (uint64_t)a.d, 32)) {
     snprintf(err, errn, "cuTensorMapEncodeTiled failed (driver entry point missing or bad pointer/shape)");
     return FEPLB_E_CUDA;
   }
@@ -534,12 +569,12 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d; p2.ab_out = nullptr;
 
-  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st)
-                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, p1, a.num_sms, st);
+  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st)
+                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st);
   ++*n_launch;
   if (e == cudaSuccess) {
-    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, p2, a.num_sms, st)
-               : launch_one<false, false>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, p2, a.num_sms, st);
+    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st)
+               : launch_one<false, false>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st);
     ++*n_launch;
   }
   if (e != cudaSuccess) {
