@@ -303,10 +303,15 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const uint32_t sa = smem_u32(smem + (size_t)stage * kStageBytes);
           const uint32_t sb = sa + kABytes;
           if (PAIR) {
-            // both CTAs credit the LEADER's barrier; the leader announces the bytes of both
+            // both CTAs credit the LEADER's barrier; the leader announces the bytes of both.  A tile
+            // whose second 128 rows hold no valid row (a group of at most 128 rows, or a ragged
+            // tail) needs no A rows in the peer: it skips that load (the MMA then multiplies
+            // whatever its stage holds into accumulator rows nobody stores), so a small group costs
+            // the pair no more operand traffic than it would cost a single CTA.
             const uint32_t full0 = map_to_cta(full, 0);
-            if (cta_rank == 0) mbar_expect_tx(full, stage_tx);
-            tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
+            const bool peer_rows = c.rows_valid > BM;
+            if (cta_rank == 0) mbar_expect_tx(full, peer_rows ? stage_tx : stage_tx - kABytes);
+            if (cta_rank == 0 || peer_rows) tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
             if (cta_rank == 0) tma_load_2d_pair(sb, mb0, full0, kb * BK, brow0);
             else tma_load_2d_pair(sb, mb1, full0, kb * BK, brow1);
           } else {
