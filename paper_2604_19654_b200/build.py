@@ -35,20 +35,34 @@ def needs_build() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    cmd = [_nvcc(), "-shared", "-O3", "-std=c++17", "-lineinfo",
-           "-gencode", "arch=compute_100a,code=sm_100a",
-           "-Xcompiler", "-fPIC,-pthread",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-    cmd[1:1] = os.environ.get("FEPLB_NVCC_FLAGS", "").split()      # e.g. -DFEPLB_GEMM_BK=32 for experiments
-    if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    r = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or r.returncode:
-        sys.stderr.write(r.stdout + r.stderr)
-    if r.returncode:
-        raise RuntimeError("nvcc failed building libfeplb.so")
-    return LIB
+    # Several processes may get here at once (one per GPU under torchrun): one builds, to a
+    # temporary name that is renamed into place, the others wait on the lock and find it done.
+    import fcntl
+    with open(LIB + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if not force and not needs_build():
+                return LIB
+            tmp = f"{LIB}.{os.getpid()}.tmp"
+            cmd = [_nvcc(), "-shared", "-O3", "-std=c++17", "-lineinfo",
+                   "-gencode", "arch=compute_100a,code=sm_100a",
+                   "-Xcompiler", "-fPIC,-pthread",
+                   "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+                   "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+            cmd[1:1] = os.environ.get("FEPLB_NVCC_FLAGS", "").split()      # e.g. -DFEPLB_GEMM_BK=32 for experiments
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            r = subprocess.run(cmd, capture_output=True, text=True)
+            if verbose or r.returncode:
+                sys.stderr.write(r.stdout + r.stderr)
+            if r.returncode:
+                if os.path.exists(tmp):
+                    os.remove(tmp)
+                raise RuntimeError("nvcc failed building libfeplb.so")
+            os.replace(tmp, LIB)
+            return LIB
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
 
 
 if __name__ == "__main__":
