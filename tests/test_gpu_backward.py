@@ -119,6 +119,36 @@ def test_backward_random_shapes(seed, monkeypatch):
     case.close()
 
 
+@pytest.mark.parametrize("pair", [0, 3])
+def test_backward_of_an_empty_batch(pair, monkeypatch):
+    """T = 0 with padded segments: every expert has zero rows.  The weight gradients are zeros when
+    overwriting and untouched when accumulating; nothing traps."""
+    import torch
+    monkeypatch.setenv("FEPLB_BWD_PAIR", str(pair))
+    w = W.get_workload("cfg1").with_(T=0)
+    cfg = F.config_from_workload(w, row_align=128)
+    ctx, buf, bwd = F.Context(cfg), F.Buffers(cfg), F.BackwardBuffers(cfg)
+    ctx.set_preact_buffer(bwd.ab)
+    z = torch.zeros(1, w.d, dtype=torch.bfloat16, device="cuda")
+    zi = torch.zeros(1, w.K, dtype=torch.int32, device="cuda")
+    zg = torch.zeros(1, w.K, device="cuda")
+    w1 = torch.ones(w.E, w.f, w.d, dtype=torch.bfloat16, device="cuda")
+    w2 = torch.ones(w.E, w.d, w.f, dtype=torch.bfloat16, device="cuda")
+    ctx.moe_forward(z, zi, zg, w1, w1, w2, buf)
+    dw1 = torch.full((w.E, w.f, w.d), 3.0, device="cuda")
+    dw3 = torch.full((w.E, w.f, w.d), 3.0, device="cuda")
+    dw2 = torch.full((w.E, w.d, w.f), 3.0, device="cuda")
+    w1t = torch.ones(w.E, w.d, w.f, dtype=torch.bfloat16, device="cuda")
+    w2t = torch.ones(w.E, w.f, w.d, dtype=torch.bfloat16, device="cuda")
+    ctx.moe_backward(z, zg, w1t, w1t, w2t, buf, bwd, dw1, dw3, dw2, accumulate=True)
+    ctx.check_status()
+    assert float(dw1.min()) == 3.0 and float(dw2.max()) == 3.0
+    ctx.moe_backward(z, zg, w1t, w1t, w2t, buf, bwd, dw1, dw3, dw2)
+    ctx.check_status()
+    assert not dw1.any() and not dw3.any() and not dw2.any()
+    ctx.close()
+
+
 def test_combine_bwd_bit_exact_rows_and_gate_gradients():
     import torch
     w = W.get_workload("cfg2").with_(T=300, E=16, R=4)
