@@ -119,6 +119,19 @@ def test_backward_random_shapes(seed, monkeypatch):
     case.close()
 
 
+def test_backward_at_the_maximum_expert_count():
+    """E = 1024: expert and group tables at the library's limit, most experts with few rows or none."""
+    w = W.get_workload("cfg2").with_(name="maxEb", T=700, E=1024, R=16, K=4, d=128, f=64, dyn=8, max_num_dyn=4, tau=1, alpha=0.3)
+    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w)
+    rdx, rdg, rdw1, rdw3, rdw2 = ref
+    _close(W.bf16_bits_to_f64(F.bf16_bits(bwd.d_x))[: w.T], rdx, "dx")
+    _close(bwd.d_gates.cpu().numpy().astype(np.float64)[: w.T], rdg, "dgates")
+    _close(dw2.cpu().numpy().astype(np.float64), rdw2, "dw2")
+    _close(dw1.cpu().numpy().astype(np.float64), rdw1, "dw1")
+    _close(dw3.cpu().numpy().astype(np.float64), rdw3, "dw3")
+    case.close()
+
+
 @pytest.mark.parametrize("pair", [0, 3])
 def test_backward_of_an_empty_batch(pair, monkeypatch):
     """T = 0 with padded segments: every expert has zero rows.  The weight gradients are zeros when

@@ -312,6 +312,16 @@ def test_forward_random_shapes(seed, monkeypatch):
     case.close()
 
 
+@pytest.mark.parametrize("A", [1, 128])
+def test_forward_at_the_maximum_expert_count(A):
+    """E = 1024 (the library's limit) on 16 ranks: group tables of 1024 entries, most experts with a
+    handful of rows or none."""
+    w = W.get_workload("cfg2").with_(name="maxE", T=1500, E=1024, R=16, K=8, d=128, f=64, dyn=8, max_num_dyn=4, tau=1, alpha=0.3)
+    case = DeviceCase(w, row_align=A)
+    _check_forward(case, sample=200)
+    case.close()
+
+
 @pytest.mark.parametrize("seed", range(4))
 def test_forward_cfg1_other_seeds(seed):
     w = W.get_workload("cfg1")
