@@ -312,6 +312,14 @@ def test_forward_random_shapes(seed, monkeypatch):
     case.close()
 
 
+def test_forward_at_the_maximum_top_k():
+    """K = 32 (the library's limit): every token goes to 32 of 64 experts."""
+    w = W.get_workload("cfg2").with_(name="maxK", T=333, E=64, R=4, K=32, d=256, f=128, dyn=4, max_num_dyn=4, tau=1)
+    case = DeviceCase(w)
+    _check_forward(case)
+    case.close()
+
+
 @pytest.mark.parametrize("A", [1, 128])
 def test_forward_at_the_maximum_expert_count(A):
     """E = 1024 (the library's limit) on 16 ranks: group tables of 1024 entries, most experts with a
