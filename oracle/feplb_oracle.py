@@ -32,6 +32,8 @@ select_dynamic  static/dynamic partition controlled by ``dyn`` (Section 2.3); a 
 expert_ffn      grouped GEMM of the experts (Sections 2.3, 3.1) with the SwiGLU expert of the
                 workload definition: y = (silu(x W1) * (x W3)) W2 in fp64.  pinned: scalar loops,
                 one-hot rows, linearity
+expert_hidden   the first half of expert_ffn on its own (h = silu(x W1) * (x W3)), which expert_ffn
+                calls; lets a test look at the CUDA path's H buffer.      pinned: through expert_ffn
 combine         "Combine phase returns results" (Section 2.3) = gate-weighted sum of the K
                 expert outputs of a token.                                pinned: K=1 round trip,
                 scalar loops
@@ -297,22 +299,33 @@ def expert_ffn(x_rows_bits: np.ndarray, row_expert: np.ndarray, w1_bits, w3_bits
     row_expert = np.asarray(row_expert)
     n = x_rows_bits.shape[0]
     d_out = w2_bits.shape[1]
+    h_all = expert_hidden(x_rows_bits, row_expert, w1_bits, w3_bits)
+    if round_h_bf16:
+        h_all = _round_f64_to_bf16(h_all)
     y = np.zeros((n, d_out), np.float64)
     for e in np.unique(row_expert).tolist():
         if e < 0:
             continue
         idx = np.flatnonzero(row_expert == e)
-        X = bf16_bits_to_f64(x_rows_bits[idx])
-        W1 = bf16_bits_to_f64(w1_bits[e])
-        W3 = bf16_bits_to_f64(w3_bits[e])
-        W2 = bf16_bits_to_f64(w2_bits[e])
-        a = X @ W1.T
-        b = X @ W3.T
-        h = silu(a) * b
-        if round_h_bf16:
-            h = _round_f64_to_bf16(h)
-        y[idx] = h @ W2.T
+        y[idx] = h_all[idx] @ bf16_bits_to_f64(w2_bits[e]).T
     return y
+
+
+def expert_hidden(x_rows_bits: np.ndarray, row_expert: np.ndarray, w1_bits, w3_bits) -> np.ndarray:
+    """The hidden activation of expert_ffn on its own: h[i,:] = silu(x_i W1[e]) * (x_i W3[e]), fp64;
+    padding rows give zeros."""
+    x_rows_bits = np.asarray(x_rows_bits)
+    row_expert = np.asarray(row_expert)
+    h = np.zeros((x_rows_bits.shape[0], w1_bits.shape[1]), np.float64)
+    for e in np.unique(row_expert).tolist():
+        if e < 0:
+            continue
+        idx = np.flatnonzero(row_expert == e)
+        X = bf16_bits_to_f64(x_rows_bits[idx])
+        a = X @ bf16_bits_to_f64(w1_bits[e]).T
+        b = X @ bf16_bits_to_f64(w3_bits[e]).T
+        h[idx] = silu(a) * b
+    return h
 
 
 def _round_f64_to_bf16(a: np.ndarray) -> np.ndarray:
