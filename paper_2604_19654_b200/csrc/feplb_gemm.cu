@@ -39,9 +39,9 @@ constexpr int kBBytesMax = 256 * BK * 2;           // 32 KiB
 //   pair (PAIR = true): a cluster of two CTAs computes a 256 x 256 tile with cta_group::2 MMAs
 //     issued by the even CTA: each CTA stages its own 128 rows of A and HALF of the B tile (the
 //     W1 tile in the even CTA and the W3 tile in the odd one in pass 1), so a CTA needs only
-//     64 bytes per MMA cycle from L2 and the ring holds 6 stages of 32 KiB.  No multicast: each
-//     CTA loads its own halves.  Used for launches whose groups are large (a 256-row tile wastes
-//     more on a ragged tail).
+//     64 bytes per MMA cycle from L2 and the ring holds 6 stages of 32 KiB.  No load is shared
+//     between the CTAs: each brings its own halves.  Used for launches whose groups are large
+//     (a 256-row tile wastes more on a ragged tail).
 // Both keep two accumulators in TMEM so that the epilogue of tile i overlaps the MMAs of tile i+1.
 template <bool PAIR> struct Ring {
   static constexpr int kStages = PAIR ? 6 : 4;
