@@ -154,6 +154,9 @@ void planner_main(feplb_ctx* c) {
         if (q != cudaErrorNotReady) { rc = FEPLB_E_CUDA; break; }
       }
       if ((spin & 1023u) == 1023u && std::chrono::duration<double>(clk::now() - w0).count() > 1e-3 * c->planner_timeout_ms) { rc = FEPLB_E_TIMEOUT; break; }
+#if defined(__x86_64__) || defined(__i386__)
+      __builtin_ia32_pause();     // a polite spin: the sibling hyper-thread (another rank's host thread) keeps its issue slots
+#endif
     }
     std::atomic_thread_fence(std::memory_order_acquire);
     c->tl.host_counts_ready_us = us_since(c->t0);
