@@ -54,6 +54,7 @@ typedef enum {
 enum { FEPLB_POLICY_LITERAL = 0, FEPLB_POLICY_FIRST_FIT = 1 };
 enum { FEPLB_MASK_GIVEN = 0, FEPLB_MASK_REACTIVE = 1 };
 enum { FEPLB_FFN_ALL = 0, FEPLB_FFN_STATIC = 1, FEPLB_FFN_DYNAMIC = 2 };
+enum { FEPLB_FORM_AUTO = -1, FEPLB_FORM_SINGLE = 0, FEPLB_FORM_PAIR = 1 };
 
 /* Layer geometry and balancer parameters.
  * Requirements: E % R == 0; d % 128 == 0; f % 64 == 0; 1 <= K <= 32; E <= 1024;
@@ -172,8 +173,8 @@ int feplb_place_experts(const double* load, int32_t E, int32_t R, int32_t* new_i
 
 /* ---- device steps ------------------------------------------------------------------------- */
 
-/* Step 0, optional (Section 2.3: "the router produces routing decisions"; Section 3.1: top-k
- * routing): top-k gating from router logits.  Per token the K largest of its E logits in
+/* Step 0, optional (Section 2.3, router; Section 3.1, top-k routing without auxiliary loss):
+ * top-k gating from router logits.  Per token the K largest of its E logits in
  * descending order, ties to the lower expert id; gates = softmax over the K selected logits
  * (fp32).  logits dev float [T,E] (finite values) -> topk_ids dev int32 [T,K], gates dev float [T,K]. */
 int feplb_route_topk(feplb_ctx* ctx, const float* logits, int32_t* topk_ids, float* gates, void* stream);
@@ -183,7 +184,7 @@ int feplb_route_topk(feplb_ctx* ctx, const float* logits, int32_t* topk_ids, flo
  * Ids outside [0,E) are skipped and raise FEPLB_E_RANGE in the status word. */
 int feplb_route_hist(feplb_ctx* ctx, const int32_t* topk_ids, int32_t* counts, int32_t* rank_load, void* stream);
 
-/* Step 3 (Section 2.2: tokens "permuted" for the grouped GEMM) = stable counting sort of the
+/* Step 3 (Section 2.2, Phase 1: rows are brought into expert order for the grouped GEMM) = stable counting sort of the
  * slots by expert id.  Slot s goes to row pad_off[e] + (earlier slots of e), with
  * pad_off[e] = sum_{e'<e} round_up(counts[e'], A).
  *   x dev bf16 [T,d], topk_ids dev [T,K], counts dev [E] (as written by feplb_route_hist)
@@ -211,7 +212,10 @@ int feplb_dispatch(feplb_ctx* ctx, const void* x, const int32_t* topk_ids, const
  *     kernels overwrite what they read before reading it).  Calls whose GPU work overlaps --
  *     other streams or threads -- race on it: serialise them.
  *   - status: dev uint32, zeroed by the caller, receives error bits (1 = expert id out of range,
- *     2 = counts disagree with topk_ids); NULL to ignore them. */
+ *     2 = counts disagree with topk_ids).  With NULL those errors cannot be detected at all (not
+ *     merely ignored): the bits go to a spare word of the shared scratch that nothing reads.  In
+ *     both cases the kernels stay inside the caller's buffers: an offending slot gets
+ *     slot_to_row = -1 and its row is not written. */
 int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, const int32_t* topk_ids,
                            const int32_t* counts, void* x_perm, int32_t* slot_to_row,
                            int32_t* row_to_token, uint32_t* status, void* stream);
@@ -223,6 +227,16 @@ int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, const int32_t
  * (same rule as feplb_select_dynamic) and also written to dyn_mask_out (dev uint8 [E], may be NULL). */
 int feplb_home_groups(feplb_ctx* ctx, const int32_t* counts, const uint8_t* dyn_mask,
                       feplb_group* groups_out, uint8_t* dyn_mask_out, void* stream);
+
+/* Expert weights enter the library output-major (w1, w3 [E,f,d]; w2 [E,d,f]) -- the only layout the
+ * GEMM entry points accept, because both operands of every contraction are then contiguous along
+ * the contracted dimension.  A caller that holds them input-major, as the operator is usually
+ * written (y = (silu(x W1) * (x W3)) W2 with W1, W3 [E,d,f] and W2 [E,f,d]), converts them once per
+ * weight update with this call: w1_in, w3_in dev bf16 [E,d,f], w2_in dev bf16 [E,f,d]
+ * -> w1, w3 dev bf16 [E,f,d], w2 dev bf16 [E,d,f] (distinct buffers).  feplb_transpose_weights below
+ * is the opposite direction (it makes the copies the backward pass reads). */
+int feplb_pack_weights(feplb_ctx* ctx, const void* w1_in, const void* w3_in, const void* w2_in,
+                       void* w1, void* w3, void* w2, void* stream);
 
 /* Steps 4-5 (Section 2.3: static-expert, then dynamic-expert grouped GEMM).  For every group g
  * in groups[0..n_groups) selected by `which` (FEPLB_FFN_ALL / _STATIC: is_dynamic == 0 /
@@ -367,6 +381,13 @@ int feplb_timeline_totals(feplb_ctx* ctx, feplb_timeline* sum, int64_t* n_forwar
  * the pending plan fails with FEPLB_E_TIMEOUT (returned by feplb_plan_wait / feplb_moe_forward) and
  * the context stays usable.  Not allowed while a plan is pending. */
 int feplb_set_planner_timeout(feplb_ctx* ctx, int32_t timeout_ms);
+/* Which form of the grouped-GEMM kernel the context uses.  forward_form: FEPLB_FORM_AUTO (default:
+ * chosen per group table from the rows per group), FEPLB_FORM_SINGLE (one CTA per 128-row tile) or
+ * FEPLB_FORM_PAIR (clusters of two CTAs on 256-row tiles) for every forward launch.
+ * backward_pair: -1 (default: chosen from the geometry) or a mask, bit 0 = activation-gradient
+ * GEMMs in the pair form, bit 1 = weight-gradient GEMMs in the pair form.  Results do not depend
+ * on the form beyond fp32 summation order.  Not allowed while a plan is pending. */
+int feplb_set_gemm_form(feplb_ctx* ctx, int32_t forward_form, int32_t backward_pair);
 /* Self-test of the device-side bounded waits: launches one thread that waits, with the routine
  * the GEMM kernels use, on an mbarrier nothing ever completes, limited to limit_us microseconds.
  * Returns FEPLB_OK if the wait gave up, raised the status bit and the kernel returned normally;

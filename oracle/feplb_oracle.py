@@ -17,7 +17,7 @@ What each function follows
 route_hist      per-expert token counts known to every device after Phase 1 (Section 2.2);
                 definition written out.                                   pinned: numpy.bincount,
                 conservation, brute force
-permute         "dynamic expert tokens are ... permuted" (Section 2.2) = stable counting sort of
+permute         the expert-order permutation of Phase 1 (Section 2.2) = stable counting sort of
                 slots by expert id; definition written out.               pinned: numpy stable
                 argsort, bijection invariants
 gather_rows     row copies of the permutation.                            pinned: round trip
@@ -34,7 +34,11 @@ expert_ffn      grouped GEMM of the experts (Sections 2.3, 3.1) with the SwiGLU 
                 one-hot rows, linearity
 expert_hidden   the first half of expert_ffn on its own (h = silu(x W1) * (x W3)), which expert_ffn
                 calls; lets a test look at the CUDA path's H buffer.      pinned: through expert_ffn
-combine         "Combine phase returns results" (Section 2.3) = gate-weighted sum of the K
+_round_f64_to_bf16  round-to-nearest-even to bf16 by way of float32 (the accumulator type of the
+                GPU path), used only by expert_ffn(round_h_bf16=True).    pinned: hand-picked ties
+                of both parities, values next to a tie, negative and tiny values, a scalar
+                integer re-implementation, the input generator's own rounding routine
+combine         the Combine phase (Section 2.3) = gate-weighted sum of the K
                 expert outputs of a token.                                pinned: K=1 round trip,
                 scalar loops
 token_straggler the paper's metric max_d T_d - mean (Section 3.1 "Metrics").  pinned: Table 3
@@ -104,7 +108,7 @@ def segment_offsets(counts, A: int = 1):
 
 
 def permute(topk_ids: np.ndarray, E: int, A: int = 1):
-    """Stable counting sort of the S slots by expert id (Section 2.2, "permuted there").
+    """Stable counting sort of the S slots by expert id (Section 2.2, Phase 1).
 
     Walking s = 0..S-1 in order, slot s goes to row pad_off[e] + (number of earlier slots of e).
     Returns (slot_to_row int64 [T,K], row_to_token int64 [S_pad] with -1 in padding rows,
@@ -160,10 +164,9 @@ def plan(counts, dyn_mask, R: int, tau: int = 0, max_num_dyn: int = 8, ranks_per
          row_align: int = 1):
     """Greedy per-micro-batch rebalancing plan (Section 2.3, load-balancer paragraph).
 
-    The paper's rule: repeatedly take the busiest dynamic expert on the most overloaded device
-    and hand it (weights and tokens) to the most underloaded device; a threshold tau keeps
-    experts with too few tokens at home; whole experts only; deterministic.  Readings where the
-    paper is silent:
+    Section 2.3 fixes the shape of the loop (source = most loaded device, object = its busiest
+    dynamic expert, target = least loaded device, a row threshold tau, whole experts, the same
+    result on every device).  Readings where it is silent:
       * load of a rank = rows ((token, k) slots) it executes, static and dynamic together;
       * most overloaded / underloaded = max / min load inside the NVLink domain, ties -> lowest
         rank id; a destination must still have a free slot in its receive buffer
@@ -329,6 +332,9 @@ def expert_hidden(x_rows_bits: np.ndarray, row_expert: np.ndarray, w1_bits, w3_b
 
 
 def _round_f64_to_bf16(a: np.ndarray) -> np.ndarray:
+    """fp64 -> float32 (numpy's round-to-nearest-even) -> bf16 (nearest, ties to the even
+    mantissa), returned as fp64.  Through float32 on purpose: the value being modelled is an fp32
+    accumulator that the kernel rounds to bf16."""
     f = a.astype(np.float32)
     u = f.view(np.uint32)
     r = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
@@ -381,8 +387,7 @@ def moe_layer(x_bits, topk_ids, gates, w1_bits, w3_bits, w2_bits, E: int, A: int
 # ----------------------------------------------------------------------------- router, placement
 
 def route_topk(logits: np.ndarray, K: int):
-    """Top-k gating (Section 2.3: "the router produces routing decisions"; Section 3.1: top-k
-    routing, no auxiliary loss): per token the K largest logits in descending order, ties to the
+    """Top-k gating (Step 0: Section 2.3, router; Section 3.1, top-k without auxiliary loss): per token the K largest logits in descending order, ties to the
     lower expert id; gates = softmax over the K selected logits.  The paper gives no formula for
     the gates; softmax over the selected logits is the workloads' definition.  PARITY UNPINNED
     against the paper; pinned against a library sort and closed forms.

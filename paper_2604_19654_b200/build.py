@@ -1,6 +1,9 @@
 """Builds libfeplb.so (C ABI + sm_100a kernels) in-tree with nvcc.
 
-``python -m paper_2604_19654_b200.build`` or ``build()``; nvcc cross-compiles without a GPU.
+``python -m paper_2604_19654_b200.build [--force] [-v] [--nvcc-flag=FLAG ...]`` or ``build()``;
+nvcc cross-compiles without a GPU.  ``-v`` prints ptxas resource usage; ``--nvcc-flag`` appends one
+extra compiler flag per occurrence (kernel experiments only; the product build takes none and
+reads no environment variable besides NVCC, the compiler's path).
 """
 from __future__ import annotations
 
@@ -32,7 +35,7 @@ def needs_build() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
     if not force and not needs_build():
         return LIB
     # Several processes may get here at once (one per GPU under torchrun): one builds, to a
@@ -49,7 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                    "-Xcompiler", "-fPIC,-pthread",
                    "-I", os.path.join(ROOT, "include"), "-I", CSRC,
                    "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
-            cmd[1:1] = os.environ.get("FEPLB_NVCC_FLAGS", "").split()      # e.g. -DFEPLB_GEMM_BK=32 for experiments
+            cmd[1:1] = list(extra_flags)
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             r = subprocess.run(cmd, capture_output=True, text=True)
@@ -66,4 +69,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                extra_flags=[a.split("=", 1)[1] for a in sys.argv if a.startswith("--nvcc-flag=")]))

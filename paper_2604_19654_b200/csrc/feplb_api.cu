@@ -37,8 +37,9 @@ struct feplb_ctx {
   char err[512] = {0};
   int64_t launches = 0;
   int gemm_pair_default = 0;   // GEMM form for launches whose group sizes the host does not know
-  int gemm_pair_forced = -1;   // FEPLB_GEMM_PAIR=0/1 forces one form everywhere (experiments, tests)
+  int gemm_pair_forced = -1;   // feplb_set_gemm_form: 0/1 forces one form everywhere, -1 = chosen per table
   int bwd_pair = 0;            // backward GEMMs in the pair form: bit 0 activation gradients, bit 1 weight gradients
+  int gemm_pair_auto = 0, bwd_pair_auto = 0;   // the choices feplb_create derived from the geometry
 
   // device scratch
   int32_t* d_block_hist = nullptr;
@@ -272,13 +273,10 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   c->num_sms = prop.multiProcessorCount;
   c->s_cap = feplb_s_pad(cfg);
   // 256-row pair tiles pay off when an expert's segment is several tiles long on average
-  c->gemm_pair_default = (int64_t)cfg->T * cfg->K >= (int64_t)2048 * cfg->E;
-  if (const char* e = getenv("FEPLB_GEMM_PAIR")) c->gemm_pair_default = c->gemm_pair_forced = atoi(e) != 0;
+  c->gemm_pair_auto = c->gemm_pair_default = (int64_t)cfg->T * cfg->K >= (int64_t)2048 * cfg->E;
   // backward GEMMs: the pair form pays once an expert's segment spans several 256-row tiles
-  // (measured: -7.5 % backward time at 1024 rows per expert, slower at 384); FEPLB_BWD_PAIR=0..3
-  // forces a choice (experiments, tests)
-  c->bwd_pair = (int64_t)cfg->T * cfg->K >= (int64_t)512 * cfg->E ? 3 : 0;
-  if (const char* e = getenv("FEPLB_BWD_PAIR")) c->bwd_pair = atoi(e) & 3;
+  // (measured: -7.5 % backward time at 1024 rows per expert, slower at 384)
+  c->bwd_pair_auto = c->bwd_pair = (int64_t)cfg->T * cfg->K >= (int64_t)512 * cfg->E ? 3 : 0;
   const int64_t S = (int64_t)cfg->T * cfg->K;
   c->nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   const int cap_moves = cfg->R * cfg->max_num_dyn;
@@ -421,7 +419,7 @@ static int dispatch_impl(feplb_ctx* c, const void* x, const int32_t* topk_ids, c
   CUDA_TRY(c, feplb_launch_permute(topk_ids, S, g.K, g.E, g.row_align, counts, c->d_block_hist, c->d_pad_off,
                                    slot_to_row, row_to_token, (int64_t)c->s_cap, c->d_status, st, &c->launches));
   CUDA_TRY(c, feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
-                                  st, &c->launches));
+                                  (int64_t)c->s_cap, c->num_sms, st, &c->launches));
   return FEPLB_OK;
 }
 
@@ -638,8 +636,8 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     cudaError_t e = feplb_launch_rank(topk_ids, S, g.K, g.E, c->d_block_hist, c->d_pad_off, slot_to_row, row_to_token,
                                       (int64_t)c->s_cap, st, &c->launches);
     if (e == cudaSuccess)
-      e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align, st,
-                              &c->launches, row_to_token, true);
+      e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
+                              (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true);
     if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "dispatch launch: %s", cudaGetErrorString(e));
   }
   TL_EVENT(EV_DISPATCH);
@@ -796,6 +794,30 @@ extern "C" int feplb_set_planner_timeout(feplb_ctx* c, int32_t timeout_ms) {
   return FEPLB_OK;
 }
 
+extern "C" int feplb_set_gemm_form(feplb_ctx* c, int32_t forward_form, int32_t backward_pair) {
+  if (!c) return FEPLB_E_INVALID;
+  if (forward_form < FEPLB_FORM_AUTO || forward_form > FEPLB_FORM_PAIR)
+    return fail(c, FEPLB_E_INVALID, "set_gemm_form: forward_form must be FEPLB_FORM_AUTO, _SINGLE or _PAIR");
+  if (backward_pair < -1 || backward_pair > 3)
+    return fail(c, FEPLB_E_INVALID, "set_gemm_form: backward_pair must be -1 (auto) or a 2-bit mask");
+  std::lock_guard<std::mutex> lk(c->mu);
+  if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "set_gemm_form: a plan is pending");
+  c->gemm_pair_forced = forward_form;
+  c->gemm_pair_default = forward_form == FEPLB_FORM_AUTO ? c->gemm_pair_auto : forward_form;
+  c->bwd_pair = backward_pair < 0 ? c->bwd_pair_auto : backward_pair;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_pack_weights(feplb_ctx* c, const void* w1_in, const void* w3_in, const void* w2_in, void* w1, void* w3,
+                                  void* w2, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  if (!w1_in || !w3_in || !w2_in || !w1 || !w3 || !w2) return fail(c, FEPLB_E_INVALID, "pack_weights: null pointer");
+  // [E,d,f] -> [E,f,d] and [E,f,d] -> [E,d,f]: the transposition of feplb_transpose_weights with d and f exchanged
+  CUDA_TRY(c, feplb_launch_transpose_weights(w1_in, w3_in, w2_in, w1, w3, w2, c->cfg.E, c->cfg.f, c->cfg.d,
+                                             (cudaStream_t)stream, &c->launches));
+  return FEPLB_OK;
+}
+
 extern "C" int feplb_selftest_bounded_wait(feplb_ctx* c, int32_t limit_us, void* stream) {
   if (!c || limit_us < 1 || limit_us > 1000000) return FEPLB_E_INVALID;
   cudaStream_t st = (cudaStream_t)stream;
@@ -816,8 +838,8 @@ extern "C" int feplb_route_topk(feplb_ctx* c, const float* logits, int32_t* topk
   if (!c) return FEPLB_E_INVALID;
   if (c->cfg.K > c->cfg.E) return fail(c, FEPLB_E_INVALID, "route_topk: K > E");
   if (c->cfg.T > 0 && (!logits || !topk_ids || !gates)) return fail(c, FEPLB_E_INVALID, "route_topk: null pointer");
-  CUDA_TRY(c, feplb_launch_route_topk(logits, c->cfg.T, c->cfg.E, c->cfg.K, topk_ids, gates, (cudaStream_t)stream,
-                                      &c->launches));
+  CUDA_TRY(c, feplb_launch_route_topk(logits, c->cfg.T, c->cfg.E, c->cfg.K, topk_ids, gates, c->num_sms,
+                                      (cudaStream_t)stream, &c->launches));
   return FEPLB_OK;
 }
 

@@ -37,8 +37,8 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
                                  cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
                                 const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token = nullptr,
-                                bool programmatic = false);
+                                int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
+                                int32_t* pad_row_to_token = nullptr, bool programmatic = false);
 // Whole-layer path: histogram + one scan kernel that emits counts, rank loads, offsets, the home
 // group table and the -1 tail of row_to_token; then the ranking alone.
 cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R, int A, int dyn,
@@ -57,7 +57,7 @@ cudaError_t feplb_launch_combine(const void* y_perm, const int32_t* slot_to_row,
                                  int T, int K, int d, int num_sms, cudaStream_t st, int64_t* n_launch);
 
 cudaError_t feplb_launch_route_topk(const float* logits, int T, int E, int K, int32_t* ids, float* gates,
-                                    cudaStream_t st, int64_t* n_launch);
+                                    int num_sms, cudaStream_t st, int64_t* n_launch);
 
 struct feplb_gemm_args {
   const void* x_perm; const void* w1; const void* w3; const void* w2;

@@ -32,23 +32,28 @@ static __device__ __align__(256) int32_t g_dispatch_scratch[kScratchInts];
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 int32_t* g_scratch_addr[kMaxDevices] = {nullptr};
+int g_num_sms[kMaxDevices] = {0};
 
 // Device address of the array on the current device.  In host code the symbol's name is only a
 // handle, never an address a kernel could use, so it is resolved through the runtime once per
 // device (with that device current) and cached.
-int scratch_for_current_device(int32_t** out) {
+int scratch_for_current_device(int32_t** out, int* num_sms) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FEPLB_E_CUDA;
   std::lock_guard<std::mutex> lk(g_mu);
   if (!g_scratch_addr[dev]) {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_dispatch_scratch) != cudaSuccess || !p) {
+    int sms = 0;
+    if (cudaGetSymbolAddress(&p, g_dispatch_scratch) != cudaSuccess || !p ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
       cudaGetLastError();
       return FEPLB_E_CUDA;
     }
+    g_num_sms[dev] = sms;
     g_scratch_addr[dev] = static_cast<int32_t*>(p);
   }
   *out = g_scratch_addr[dev];
+  *num_sms = g_num_sms[dev];
   return FEPLB_OK;
 }
 
@@ -68,7 +73,8 @@ extern "C" int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, co
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(x_perm)) & 15u) return FEPLB_E_INVALID;
   }
   int32_t* scratch = nullptr;
-  if ((rc = scratch_for_current_device(&scratch)) != FEPLB_OK) return rc;
+  int num_sms = 0;
+  if ((rc = scratch_for_current_device(&scratch, &num_sms)) != FEPLB_OK) return rc;
   int32_t* block_hist = scratch;
   int32_t* pad_off = scratch + kMaxHist;
   uint32_t* st_word = status ? status : reinterpret_cast<uint32_t*>(scratch + kMaxHist + FEPLB_MAX_EXPERTS + 1);
@@ -80,7 +86,7 @@ extern "C" int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, co
                            row_to_token, s_cap, st_word, st, &launches) != cudaSuccess)
     return FEPLB_E_CUDA;
   if (feplb_launch_gather(x, slot_to_row, counts, pad_off, x_perm, cfg->T, cfg->K, cfg->E, cfg->d, cfg->row_align,
-                          st, &launches) != cudaSuccess)
+                          s_cap, num_sms, st, &launches) != cudaSuccess)
     return FEPLB_E_CUDA;
   return FEPLB_OK;
 }

@@ -1,6 +1,6 @@
 // Integer side of the FEPLB hot path on sm_100a: routing histogram (paper Section 2.2: per-expert
 // token counts known after Phase 1), the stable counting-sort permutation of (token, k) slots
-// into expert-contiguous rows (Section 2.2: tokens "permuted" for the grouped GEMM), the row
+// into expert-contiguous rows (Section 2.2, Phase 1: expert order for the grouped GEMM), the row
 // gather, and the home (pre-plan) group table the static-expert GEMM runs on (Section 2.3).
 //
 // Ranks inside an expert's segment must not depend on the order in which atomics land, so
@@ -91,38 +91,43 @@ k_block_hist(const int32_t* __restrict__ ids, int64_t S, int E, int L, int32_t* 
   }
 }
 
-// Block-wide exclusive scan of v over threads 0..n-1 (n <= 1024 = blockDim.x); tmp holds 1024+32 ints.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* tmp, int* total) {
+// Block-wide exclusive scan of v over the 1024 threads of the block; tmp holds 64 values.
+template <typename V = int>
+__device__ __forceinline__ V block_exclusive_scan(V v, V* tmp, V* total) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  int x = v;
+  V x = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    int y = __shfl_up_sync(0xffffffffu, x, o);
+    V y = __shfl_up_sync(0xffffffffu, x, o);
     if (lane >= o) x += y;
   }
   if (lane == 31) tmp[w] = x;
   __syncthreads();
   if (w == 0) {
-    int s = tmp[lane];
+    V s = tmp[lane];
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int y = __shfl_up_sync(0xffffffffu, s, o);
+      V y = __shfl_up_sync(0xffffffffu, s, o);
       if (lane >= o) s += y;
     }
     tmp[32 + lane] = s;   // inclusive scan of the warp sums
   }
   __syncthreads();
-  const int warp_off = w ? tmp[32 + w - 1] : 0;
+  const V warp_off = w ? tmp[32 + w - 1] : 0;
   if (total) *total = tmp[32 + 31];
   return warp_off + x - v;
 }
 
 // Exclusive scan of the per-CTA histograms over CTAs (in place), check against counts, and
 // pad_off[e] = sum_{e'<e} round_up(counts[e'], A); pad_off[E] = padded total.
+// The counts are the caller's: when they disagree with the ids (FEPLB_ST_COUNTS) the result is
+// wrong but every later access stays inside the caller's buffers -- a negative count is taken as
+// zero, offsets are summed in 64 bits and clamped to s_cap, a padded total beyond s_cap is reported;
+// k_rank then drops the rows that do not fit.
 __global__ void __launch_bounds__(1024)
 k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __restrict__ counts,
-       int32_t* __restrict__ pad_off, uint32_t* status) {
-  __shared__ int tmp[64];
+       int32_t* __restrict__ pad_off, int64_t s_cap, uint32_t* status) {
+  __shared__ long long tmp[64];
   const int e = threadIdx.x;
   int c = 0;
   if (e < E) {
@@ -134,12 +139,15 @@ k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __
     }
     c = counts[e];
     if (run != c) atomicOr(status, FEPLB_ST_COUNTS);
+    if (c < 0) c = 0;
   }
-  const int padded = (c + A - 1) / A * A;
-  int total;
-  const int off = block_exclusive_scan(padded, tmp, &total);
-  if (e < E) pad_off[e] = off;
-  if (e == 0) pad_off[E] = total;
+  long long total;
+  const long long off = block_exclusive_scan<long long>(((long long)c + A - 1) / A * A, tmp, &total);
+  if (e < E) pad_off[e] = (int32_t)(off < s_cap ? off : s_cap);
+  if (e == 0) {
+    pad_off[E] = (int32_t)(total < s_cap ? total : s_cap);
+    if (total > s_cap) atomicOr(status, FEPLB_ST_COUNTS);
+  }
 }
 
 // Whole-layer variant of k_scan: from the per-CTA histograms alone it produces everything the
@@ -243,8 +251,9 @@ k_rank(const int32_t* __restrict__ ids, int64_t S, int K, int E, const int32_t* 
     if (v >= 0 && lane == __ffs(mk[c]) - 1) wh[w * E + v] += __popc(mk[c]);
     __syncwarp();
     if (s < S) {
+      if (row >= s_cap) row = -1;      // only with counts that disagree with the ids (reported by the scan)
       slot_to_row[s] = row;
-      if (row >= 0 && row < s_cap) row_to_token[row] = (int32_t)(s / K);
+      if (row >= 0) row_to_token[row] = (int32_t)(s / K);
     }
   }
 }
@@ -302,10 +311,16 @@ k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, u
 // Zero the padding rows at the end of every expert's segment (row_align > 1 only).
 __global__ void __launch_bounds__(kThreads)
 k_zero_pad(const int32_t* __restrict__ counts, const int32_t* __restrict__ pad_off, uint4* __restrict__ x_perm,
-           int chunks, int32_t* __restrict__ row_to_token) {
+           int chunks, int32_t* __restrict__ row_to_token, int64_t s_cap) {
   pdl_sync();
   const int e = blockIdx.x;
-  const int64_t r0 = (int64_t)pad_off[e] + counts[e], r1 = pad_off[e + 1];
+  // clamped to the buffer: counts that disagree with the ids must not turn into wild writes
+  const int c = counts[e] > 0 ? counts[e] : 0;
+  int64_t r1 = pad_off[e + 1];
+  if (r1 > s_cap) r1 = s_cap;
+  int64_t r0 = (int64_t)pad_off[e] + c;
+  if (r0 > r1) r0 = r1;
+  if (r0 < 0) r0 = 0;
   if (row_to_token)
     for (int64_t r = r0 + threadIdx.x; r < r1; r += kThreads) row_to_token[r] = -1;
   const int64_t n = (r1 - r0) * chunks;
@@ -323,7 +338,7 @@ k_home_groups(const int32_t* __restrict__ counts, const uint8_t* __restrict__ ma
   const int e = threadIdx.x;
   const int c = e < E ? counts[e] : 0;
   if (e < E) sc[e] = c;
-  const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, nullptr);
+  const int off = block_exclusive_scan<int>((c + A - 1) / A * A, tmp, nullptr);
   if (e >= E) return;
   int is_dyn;
   if (mask_in) {
@@ -417,7 +432,7 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
     ++*n_launch;
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
   }
-  k_scan<<<1, 1024, 0, st>>>(block_hist, nb, E, A, counts, pad_off, status);
+  k_scan<<<1, 1024, 0, st>>>(block_hist, nb, E, A, counts, pad_off, s_cap, status);
   ++*n_launch;
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   if (nb) {
@@ -430,17 +445,19 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
 
 cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
                                 const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                cudaStream_t st, int64_t* n_launch, int32_t* pad_row_to_token, bool programmatic) {
+                                int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
+                                int32_t* pad_row_to_token, bool programmatic) {
   cudaError_t err;
   const int chunks = d / 8;
   if (A > 1) {
-    err = launch(k_zero_pad, E, kThreads, 0, st, programmatic, counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token);
+    err = launch(k_zero_pad, E, kThreads, 0, st, programmatic, counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token,
+                 s_cap);
     ++*n_launch;
     if (err != cudaSuccess) return err;
   }
   if (T == 0) return cudaSuccess;
   const int64_t units = (int64_t)T * ((chunks + 32 * kGatherUnroll - 1) / (32 * kGatherUnroll));
-  int blocks = 148 * 8;   // 8 CTAs of 256 threads per SM are resident
+  int blocks = num_sms * 8;   // 8 CTAs of 256 threads per SM are resident
   const int64_t need = (units + kWarps - 1) / kWarps;
   if (need < blocks) blocks = (int)need;
   ++*n_launch;
@@ -498,10 +515,10 @@ cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const
 }
 
 cudaError_t feplb_launch_route_topk(const float* logits, int T, int E, int K, int32_t* ids, float* gates,
-                                    cudaStream_t st, int64_t* n_launch) {
+                                    int num_sms, cudaStream_t st, int64_t* n_launch) {
   if (T == 0) return cudaSuccess;
   int blocks = (T + kWarps - 1) / kWarps;
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > num_sms * 8) blocks = num_sms * 8;
   const int nper = (E + 31) / 32;
   ++*n_launch;
   if (nper <= 1) k_route_topk<1><<<blocks, kThreads, 0, st>>>(logits, T, E, K, ids, gates);

@@ -19,6 +19,7 @@ OK, E_INVALID, E_RANGE, E_CUDA, E_NOMEM, E_TIMEOUT, E_STATE, E_DEVICE = 0, -1, -
 POLICY_LITERAL, POLICY_FIRST_FIT = 0, 1
 MASK_GIVEN, MASK_REACTIVE = 0, 1
 FFN_ALL, FFN_STATIC, FFN_DYNAMIC = 0, 1, 2
+FORM_AUTO, FORM_SINGLE, FORM_PAIR = -1, 0, 1
 HOST_SLOTS = 4            # staging sets of the pipelined host-buffer forward (FEPLB_HOST_SLOTS)
 
 
@@ -106,6 +107,8 @@ def lib() -> C.CDLL:
             "feplb_dispatch_bwd": (C.c_int, [vp] * 5),
             "feplb_moe_backward": (C.c_int, [vp] * 19 + [i32, vp]),
             "feplb_set_planner_timeout": (C.c_int, [vp, i32]),
+            "feplb_set_gemm_form": (C.c_int, [vp, i32, i32]),
+            "feplb_pack_weights": (C.c_int, [vp] * 8),
             "feplb_selftest_bounded_wait": (C.c_int, [vp, i32, vp]),
             "feplb_launch_count": (i64, [vp]),
         }
@@ -401,6 +404,15 @@ class Context:
             _ptr(buf.h_scratch), _ptr(buf.y_perm), _ptr(buf.slot_to_row), _ptr(bwd.d_y_perm),
             _ptr(bwd.d_ab), _ptr(bwd.d_x_perm), _ptr(bwd.d_x), _ptr(bwd.d_gates), _ptr(dw1),
             _ptr(dw3), _ptr(dw2), int(bool(accumulate)), self._stream(stream)), "feplb_moe_backward")
+
+    def set_gemm_form(self, forward_form: int = FORM_AUTO, backward_pair: int = -1):
+        """Forces the grouped-GEMM form (FORM_*) of the forward launches and the pair mask of the backward GEMMs."""
+        self._chk(lib().feplb_set_gemm_form(self._h, int(forward_form), int(backward_pair)), "feplb_set_gemm_form")
+
+    def pack_weights(self, w1_in, w3_in, w2_in, w1, w3, w2, stream=None):
+        """Input-major weights ([E,d,f], [E,d,f], [E,f,d]) -> the library's output-major layout."""
+        self._chk(lib().feplb_pack_weights(self._h, _ptr(w1_in), _ptr(w3_in), _ptr(w2_in), _ptr(w1), _ptr(w3), _ptr(w2),
+                                           self._stream(stream)), "feplb_pack_weights")
 
     def set_planner_timeout(self, timeout_ms: int):
         self._chk(lib().feplb_set_planner_timeout(self._h, int(timeout_ms)), "feplb_set_planner_timeout")

@@ -14,6 +14,8 @@ from paper_2604_19654_b200 import build as B
 from paper_2604_19654_b200 import feplb as F
 from paper_2604_19654_b200 import workloads as W
 
+from golden_utils import load_plan_cases
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -91,6 +93,33 @@ def test_plan_matches_oracle_bit_exact(R, L, seed, tau, mnd, policy, split, g, d
     cfg = F.make_config(T=1, K=1, E=E, R=R, d=128, f=64, max_num_dyn=mnd, tau=tau, ranks_per_domain=D,
                         policy=policy, split=split, split_granule=g, row_align=A)
     _same_plan(cfg, counts, mask, A)
+
+
+@pytest.mark.parametrize("c", load_plan_cases(), ids=lambda c: c["case"])
+def test_c_planner_against_the_handworked_plans(c):
+    """feplb_plan (the library's C++ planner) against the hand-worked file itself, not through the
+    oracle: the two planners follow the same reading, so agreement between them proves nothing
+    about branches both could misread."""
+    R, L = int(c["R"]), int(c["L"])
+    cfg = F.make_config(T=1, K=1, E=R * L, R=R, d=128, f=64, max_num_dyn=int(c["max_num_dyn"]), tau=int(c["tau"]),
+                        ranks_per_domain=int(c["domain"]),
+                        policy=F.POLICY_LITERAL if c["policy"] == "literal" else F.POLICY_FIRST_FIT,
+                        split=int(c["split"]), split_granule=int(c["g"]))
+    p = F.plan(cfg, np.array(c["counts_i"], np.int32), np.array(c["mask_i"], np.uint8))
+    assert p.moves == c["moves_t"]
+    assert p.load_before.tolist() == c["before_i"] and p.load_after.tolist() == c["after_i"]
+    # the group table follows from the moves: pieces from the front of the segment, then the rest
+    off, exp = 0, []
+    for e, cnt in enumerate(c["counts_i"]):
+        pos, left = off, cnt
+        for (me, _s, dst, rows) in c["moves_t"]:
+            if me == e:
+                exp.append((e, pos, rows, dst, c["mask_i"][e]))
+                pos, left = pos + rows, left - rows
+        if left > 0:
+            exp.append((e, pos, left, e // L, c["mask_i"][e]))
+        off += cnt
+    assert p.groups == exp
 
 
 def test_plan_matches_oracle_on_workloads():

@@ -41,11 +41,12 @@ def test_transpose_weights_bit_exact():
     case.close()
 
 
-def _run_backward(w, mb=0, scale=1.0, **cfg_kw):
+def _run_backward(w, mb=0, scale=1.0, pair=-1, **cfg_kw):
     import torch
     case = DeviceCase(w, mb=mb, row_align=128, **cfg_kw)
     bwd = F.BackwardBuffers(case.cfg)
     ctx = case.ctx
+    ctx.set_gemm_form(F.FORM_AUTO, pair)
     ctx.set_preact_buffer(bwd.ab)
     ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
     w1t = torch.zeros(w.E, w.d, w.f, dtype=torch.bfloat16, device="cuda")
@@ -65,15 +66,14 @@ def _run_backward(w, mb=0, scale=1.0, **cfg_kw):
 
 @pytest.mark.parametrize("pair", [0, 3])
 @pytest.mark.parametrize("name,T", [("cfg1", 256), ("cfg2", 384), ("cfg4", 512)])
-def test_backward_parity(name, T, pair, monkeypatch):
+def test_backward_parity(name, T, pair):
     """``pair``: both forms of the backward GEMMs (single CTA per 128-row tile; clusters of two CTAs on
-    256-row tiles), forced through the environment switch the context reads when it is created."""
+    256-row tiles), forced with feplb_set_gemm_form."""
     import torch
-    monkeypatch.setenv("FEPLB_BWD_PAIR", str(pair))
     w = W.get_workload(name).with_(T=T)
     if name != "cfg1":
         w = w.with_(E=16, R=4)                       # fewer experts: the fp64 reference stays cheap
-    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w)
+    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w, pair=pair)
     rdx, rdg, rdw1, rdw3, rdw2 = ref
     _close(W.bf16_bits_to_f64(F.bf16_bits(bwd.d_x))[: w.T], rdx, "dx")
     _close(bwd.d_gates.cpu().numpy().astype(np.float64)[: w.T], rdg, "dgates")
@@ -97,7 +97,7 @@ def test_backward_parity(name, T, pair, monkeypatch):
 
 
 @pytest.mark.parametrize("seed", range(8))
-def test_backward_random_shapes(seed, monkeypatch):
+def test_backward_random_shapes(seed):
     """Seeded random small layers (odd token counts, 1-4 ranks, ragged tiles, experts without rows),
     both GEMM forms."""
     rng = np.random.default_rng(9100 + seed)
@@ -108,8 +108,7 @@ def test_backward_random_shapes(seed, monkeypatch):
         name=f"randb{seed}", T=int(rng.integers(1, 500)), E=E, R=R, K=int(rng.integers(1, min(E, 6) + 1)),
         d=int(rng.choice([128, 256, 384])), f=int(rng.choice([64, 192, 256])), dyn=int(rng.integers(0, L + 1)),
         max_num_dyn=2, tau=8, routing="dirichlet", alpha=float(rng.choice([0.1, 0.5])))
-    monkeypatch.setenv("FEPLB_BWD_PAIR", str(int(rng.choice([0, 3]))))
-    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w, mb=seed)
+    case, bwd, (dw1, dw3, dw2), ref, wt, d_out = _run_backward(w, mb=seed, pair=int(rng.choice([0, 3])))
     rdx, rdg, rdw1, rdw3, rdw2 = ref
     _close(W.bf16_bits_to_f64(F.bf16_bits(bwd.d_x))[: w.T], rdx, "dx")
     _close(bwd.d_gates.cpu().numpy().astype(np.float64)[: w.T], rdg, "dgates")
@@ -133,14 +132,14 @@ def test_backward_at_the_maximum_expert_count():
 
 
 @pytest.mark.parametrize("pair", [0, 3])
-def test_backward_of_an_empty_batch(pair, monkeypatch):
+def test_backward_of_an_empty_batch(pair):
     """T = 0 with padded segments: every expert has zero rows.  The weight gradients are zeros when
     overwriting and untouched when accumulating; nothing traps."""
     import torch
-    monkeypatch.setenv("FEPLB_BWD_PAIR", str(pair))
     w = W.get_workload("cfg1").with_(T=0)
     cfg = F.config_from_workload(w, row_align=128)
     ctx, buf, bwd = F.Context(cfg), F.Buffers(cfg), F.BackwardBuffers(cfg)
+    ctx.set_gemm_form(F.FORM_AUTO, pair)
     ctx.set_preact_buffer(bwd.ab)
     z = torch.zeros(1, w.d, dtype=torch.bfloat16, device="cuda")
     zi = torch.zeros(1, w.K, dtype=torch.int32, device="cuda")

@@ -99,6 +99,45 @@ def test_dispatch_with_wrong_counts_is_reported():
     ctx.close()
 
 
+@pytest.mark.parametrize("A", [1, 128])
+@pytest.mark.parametrize("noalloc", [False, True])
+def test_dispatch_with_wrong_counts_stays_inside_the_buffers(A, noalloc):
+    """Counts that disagree with the ids (too large, too small, negative, absurdly large) give a wrong
+    permutation and FEPLB_E_DEVICE, but no access outside x_perm / row_to_token: both are
+    allocated with guard rows behind them that must stay untouched, and every slot_to_row entry is
+    -1 or a row inside the buffer."""
+    torch = _torch()
+    w = _tiny(64, 2, 8, 2)
+    cfg = F.config_from_workload(w, row_align=A)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    cap, guard = F.s_pad(cfg), 64
+    ids = np.random.default_rng(0).integers(0, 8, size=(w.T, w.K)).astype(np.int32)
+    d_ids = torch.from_numpy(ids).cuda()
+    d_x = F.bf16_tensor(W.gen_activations(w, 0))
+    true_counts = np.bincount(ids.ravel(), minlength=w.E).astype(np.int32)
+    for delta in ({3: +1}, {7: +5}, {0: -2}, {2: -10 ** 6}, {1: 2 ** 30, 2: 2 ** 30, 3: 2 ** 30}, {5: +1000}):
+        counts = true_counts.copy()
+        for e, dv in delta.items():
+            counts[e] = dv if abs(dv) >= 10 ** 6 else counts[e] + dv
+        xp = torch.full((cap + guard, w.d), 9.0, dtype=torch.bfloat16, device="cuda")
+        r2t = torch.full((cap + guard,), 12345, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        d_counts = torch.from_numpy(counts).cuda()
+        if noalloc:
+            F.dispatch_noalloc(cfg, d_x, d_ids, d_counts, xp, buf.slot_to_row, r2t, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) & 2
+        else:
+            ctx.dispatch(d_x, d_ids, d_counts, xp, buf.slot_to_row, r2t)
+            with pytest.raises(F.FeplbError) as ei:
+                ctx.check_status()
+            assert ei.value.code == F.E_DEVICE
+        assert bool((xp[cap:] == 9.0).all()) and bool((r2t[cap:] == 12345).all()), delta
+        s2r = buf.slot_to_row.cpu().numpy()
+        assert ((s2r >= -1) & (s2r < cap)).all(), delta
+    ctx.close()
+
+
 def test_home_groups_match_the_no_move_plan():
     torch = _torch()
     for w, A in ((W.get_workload("cfg2"), 1), (W.get_workload("cfg1"), 128)):
@@ -329,10 +368,10 @@ def _random_workload(seed):
 
 
 @pytest.mark.parametrize("seed", range(16))
-def test_forward_random_shapes(seed, monkeypatch):
+def test_forward_random_shapes(seed):
     w, A, split, pair = _random_workload(seed)
-    monkeypatch.setenv("FEPLB_GEMM_PAIR", str(pair))
     case = DeviceCase(w, mb=seed, row_align=A, split=split, split_granule=128 if A == 128 else 16)
+    case.ctx.set_gemm_form(F.FORM_PAIR if pair else F.FORM_SINGLE)
     _check_forward(case)
     case.close()
 

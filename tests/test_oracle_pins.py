@@ -11,6 +11,8 @@ from hypothesis import given, settings, strategies as st
 from oracle import feplb_oracle as O
 from paper_2604_19654_b200 import workloads as W
 
+from golden_utils import load_plan_cases
+
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
@@ -129,39 +131,17 @@ def test_gather_rows_roundtrip():
 
 # ----------------------------------------------------------------------------- plan
 
-def _load_cases():
-    cases, cur = [], None
-    for line in open(os.path.join(GOLDEN, "plan_handworked.txt")):
-        line = line.split("#")[0].rstrip("\n")
-        if "=" not in line:
-            continue
-        k, v = [s.strip() for s in line.split("=", 1)]
-        if k == "case":
-            cur = {"case": v}
-            cases.append(cur)
-        else:
-            cur[k] = v
-    return cases
-
-
-@pytest.mark.parametrize("c", _load_cases(), ids=lambda c: c["case"])
+@pytest.mark.parametrize("c", load_plan_cases(), ids=lambda c: c["case"])
 def test_plan_handworked(c):
     R, L = int(c["R"]), int(c["L"])
-    counts = [int(v) for v in c["counts"].split()]
-    mask = [int(v) for v in c["mask"].split()]
-    p = O.plan(counts, mask, R, tau=int(c["tau"]), max_num_dyn=int(c["max_num_dyn"]),
+    p = O.plan(c["counts_i"], c["mask_i"], R, tau=int(c["tau"]), max_num_dyn=int(c["max_num_dyn"]),
                ranks_per_domain=int(c["domain"]),
                policy=O.POLICY_LITERAL if c["policy"] == "literal" else O.POLICY_FIRST_FIT,
                split=int(c["split"]), split_granule=int(c["g"]))
-    exp_moves = []
-    for m in c["moves"].split():
-        e, sd, rows = m.split(":")
-        s, dd = sd.split(">")
-        exp_moves.append((int(e), int(s), int(dd), int(rows)))
-    assert p["moves"] == exp_moves
-    assert p["load_before"].tolist() == [int(v) for v in c["load_before"].split()]
-    assert p["load_after"].tolist() == [int(v) for v in c["load_after"].split()]
-    assert len(counts) == R * L
+    assert p["moves"] == c["moves_t"]
+    assert p["load_before"].tolist() == c["before_i"]
+    assert p["load_after"].tolist() == c["after_i"]
+    assert len(c["counts_i"]) == R * L
 
 
 def _check_plan_invariants(counts, mask, R, p, tau, max_num_dyn, D, split, g, A=1):
@@ -400,6 +380,76 @@ def test_ffn_one_hot_rows_and_linearity():
     y2 = O.expert_ffn(xr, np.zeros(4, int), w1, w3, _bits(2 * W.bf16_bits_to_f32(w2)))
     assert np.allclose(y2, 2 * y1, rtol=1e-12)
     assert not O.expert_ffn(xr, np.zeros(4, int), w1, np.zeros_like(w3), w2).any()
+
+
+def _rne_bf16_scalar(v: float) -> float:
+    """Round one double to bf16 the way the hidden activation is stored: first to float32 (the
+    accumulator's type), then to the nearest bf16, ties to the even mantissa -- written with
+    integer arithmetic on the float32 bit pattern, one value at a time."""
+    import struct
+    (u,) = struct.unpack("<I", struct.pack("<f", v))          # struct rounds the double to float32
+    keep, drop = u >> 16, u & 0xFFFF
+    if drop > 0x8000 or (drop == 0x8000 and (keep & 1)):
+        keep += 1
+    (out,) = struct.unpack("<f", struct.pack("<I", (keep << 16) & 0xFFFFFFFF))
+    return float(out)
+
+
+def test_bf16_rounding_of_the_hidden_activation_is_nearest_even():
+    """Pins oracle._round_f64_to_bf16 (the round_h_bf16 mode of expert_ffn) on values whose bf16
+    neighbours are known by hand: bf16 keeps 8 significant bits, so the spacing at 1.0 is 2^-7."""
+    r = lambda v: float(O._round_f64_to_bf16(np.array([v], np.float64))[0])
+    assert r(1.0) == 1.0
+    assert r(1.0 + 2.0 ** -8) == 1.0                            # tie -> even mantissa (down)
+    assert r(1.0 + 3 * 2.0 ** -8) == 1.0 + 2.0 ** -6             # tie -> even mantissa (up)
+    assert r(1.0 + 2.0 ** -8 + 2.0 ** -20) == 1.0 + 2.0 ** -7    # just above the tie
+    assert r(1.0 + 2.0 ** -8 - 2.0 ** -20) == 1.0                # just below it (truncation would also
+    assert r(1.0 + 2.0 ** -7 - 2.0 ** -20) == 1.0 + 2.0 ** -7    #  give 1.0 here, but not on this line)
+    assert r(-(1.0 + 3 * 2.0 ** -8)) == -(1.0 + 2.0 ** -6)       # sign-symmetric
+    assert r(-(1.0 + 2.0 ** -8)) == -1.0
+    assert r(2.0 ** -100 * (1.0 + 2.0 ** -8 + 2.0 ** -9)) == 2.0 ** -100 * (1.0 + 2.0 ** -7)   # small normal value
+    assert r(255.5) == 256.0 and r(254.5) == 254.0 and r(0.0) == 0.0   # carry into the exponent; 254.5 ties to even
+    # the value passes through float32 first, as the kernel's fp32 accumulator does: 2^-30 is below
+    # float32's resolution at 1.0, so this is the tie again, not "just above" it
+    assert r(1.0 + 2.0 ** -8 + 2.0 ** -30) == 1.0
+    # on values that are exact in float32 it is the input generator's rounding (a separate routine)
+    rng = np.random.default_rng(12)
+    v32 = (rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, size=4096)).astype(np.float32)
+    v32[:8] = np.float32(1.0) + np.arange(8, dtype=np.float32) * np.float32(2.0 ** -8)     # ties of both parities
+    got = O._round_f64_to_bf16(v32.astype(np.float64))
+    assert np.array_equal(got, W.bf16_bits_to_f64(W.f32_to_bf16_bits(v32)))
+    assert np.array_equal(got, np.array([_rne_bf16_scalar(float(v)) for v in v32]))
+
+
+def test_ffn_with_rounded_hidden_activation_against_scalar_loops():
+    """expert_ffn(round_h_bf16=True): the hidden activation is rounded to bf16 before the second
+    contraction.  Checked against scalar loops with the rounding written out per element."""
+    rng = np.random.default_rng(13)
+    E, d, f, n = 2, 6, 5, 6
+    x = _bits(rng.standard_normal((n, d)))
+    w1 = _bits(rng.standard_normal((E, f, d)))
+    w3 = _bits(rng.standard_normal((E, f, d)))
+    w2 = _bits(rng.standard_normal((E, d, f)))
+    re = np.array([1, 0, 0, -1, 1, 0])
+    y = O.expert_ffn(x, re, w1, w3, w2, round_h_bf16=True)
+    y_plain = O.expert_ffn(x, re, w1, w3, w2)
+    X, W1, W3, W2 = (W.bf16_bits_to_f64(a) for a in (x, w1, w3, w2))
+    changed = 0
+    for i in range(n):
+        e = re[i]
+        if e < 0:
+            assert not y[i].any()
+            continue
+        h = []
+        for c in range(f):
+            a = sum(X[i, j] * W1[e, c, j] for j in range(d))
+            b = sum(X[i, j] * W3[e, c, j] for j in range(d))
+            h.append(_rne_bf16_scalar(a / (1.0 + math.exp(-a)) * b))
+        for o in range(d):
+            ref = sum(h[c] * W2[e, o, c] for c in range(f))
+            assert y[i, o] == pytest.approx(ref, rel=1e-12, abs=1e-15)
+            changed += y[i, o] != y_plain[i, o]
+    assert changed > 0                                          # the mode really rounds something
 
 
 # ----------------------------------------------------------------------------- combine, whole layer
