@@ -31,7 +31,10 @@ METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 # DRAM bytes (read + write) of one k_grouped_gemm launch at the benchmarked workload, from the ncu
 # capture summarised under profiles/; None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 190.0e6}   # profiles/k_grouped_gemm_cfg2.md: 760 MB over the 4 launches
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    "cfg2": {"bytes": 190.0e6, "source": "profiles/k_grouped_gemm_cfg2.md: 760 MB over the 4 launches of one forward"},
+}
+FFN_LAUNCHES_PER_FORWARD = 4    # static pass 1 / pass 2, dynamic pass 1 / pass 2
 
 
 def _peaks():
@@ -68,17 +71,26 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def mark(self):
+        """Index of the next sample: ``summary(a, b)`` then covers what was sampled between two marks."""
+        time.sleep(0.06)                       # let the sample that covers "now" arrive
+        return len(self.lines)
+
     def stop(self):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+        return self.summary(0, None)
+
+    def summary(self, a=0, b=None):
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            self.proc.kill()
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
         sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        for ln in self.lines[a:b]:
             f = [s.strip() for s in ln.split(",")]
             if len(f) < 9:
                 continue
@@ -250,25 +262,43 @@ def run_cuda(args, w):
             step(i)
         ev1.record(stream)
         barrier()
-        return ev0.elapsed_time(ev1)
+        return max_over_ranks(ev0.elapsed_time(ev1), world, "cuda")
+
+    def timed_blocks(min_total_ms):
+        """Blocks of exactly K steps, each bracketed by barrier + synchronize and timed by CUDA events
+        on the launching stream (slowest rank), repeated until the timed region is long enough for
+        the clock samples to mean something; the median block is reported."""
+        blocks = []
+        while len(blocks) < args.max_repeats and (not blocks or sum(blocks) < min_total_ms):
+            blocks.append(timed(args.steps))
+        return blocks
 
     # (1) the headline: K steps between two events, nothing else on the stream
+    m0 = sampler.mark() if rank == 0 else 0
     launches0 = ctx.launch_count()
-    ms_total = timed(args.steps)
-    launches = ctx.launch_count() - launches0
+    blocks = timed_blocks(args.min_timed_ms)
+    launches = (ctx.launch_count() - launches0) // len(blocks)
+    m1 = sampler.mark() if rank == 0 else 0
     ctx.check_status()
-    # (2) the same K steps again with the library's per-stage events on (they end each stage's
+    ms_total = float(np.median(blocks))
+    args.repeats, args.block_ms_min, args.block_ms_max = len(blocks), float(min(blocks)), float(max(blocks))
+    # (2) the same blocks again with the library's per-stage events on (they end each stage's
     # chain of programmatic launches, so this pass is slower): stage times and the kernel roofline
     ctx.set_timeline(True)
     ctx.timeline_totals(reset=True)
-    ms_instr = timed(args.steps)
+    blocks2 = timed_blocks(args.min_timed_ms)
     totals, n_fw = ctx.timeline_totals(reset=True)
     ctx.set_timeline(False)
-    clocks = sampler.stop() if rank == 0 else None
+    m2 = sampler.mark() if rank == 0 else 0
     ctx.check_status()
-    ms_total = max_over_ranks(ms_total, world, "cuda")
-    args.ms_instrumented = max_over_ranks(ms_instr, world, "cuda") / args.steps
+    clocks = sampler.summary(m0, m1) if rank == 0 else None
+    args.clocks_stage_pass = sampler.summary(m1, m2) if rank == 0 else None
+    args.ms_instrumented = float(np.median(blocks2)) / args.steps
     value = whole_job_throughput(world, args.steps, w.T, ms_total)
+    # (3) dispatch and combine alone over rotating buffer sets larger than the L2 (cold figures)
+    args.cold = measure_cold_io(F, ctx, cfg, w, dev, stream) if rank == 0 and not args.quick else None
+    if rank == 0:
+        sampler.stop()
 
     # ---- end to end through the host-buffer entry point -----------------------------------------
     e2e_value, h2d, d2h = None, w.T * w.d * 2 + 2 * w.T * w.K * 4, w.T * w.d * 2
@@ -286,6 +316,84 @@ def run_cuda(args, w):
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def measure_cold_io(F, ctx, cfg, w, dev, stream, reps=24):
+    """feplb_dispatch and feplb_combine timed alone, each call on the next of several buffer sets
+    whose combined footprint exceeds the 126 MB L2, so that neither the rows read nor the rows
+    written are still cached from the previous call.  Median of CUDA-event times per call."""
+    import torch
+    per_set = 2.0 * (w.T * w.d + 2 * w.S * w.d)                  # x, x_perm, y_perm of one set
+    n_sets = int(min(8, max(3, np.ceil(3 * 126e6 / per_set) + 1)))
+    sets = [F.Buffers(cfg) for _ in range(n_sets)]
+    n_mb = len(dev)
+    for i, b in enumerate(sets):                                  # fill every set once (valid indices, y_perm defined)
+        x, ids, g = dev[i % n_mb]
+        ctx.route_hist(ids, b.counts, b.rank_load, stream=stream)
+        ctx.dispatch(x, ids, b.counts, b.x_perm, b.slot_to_row, b.row_to_token, stream=stream)
+        b.y_perm.copy_(b.x_perm)
+    torch.cuda.synchronize()
+    ctx.check_status()
+    t_disp, t_comb = [], []
+    for r in range(reps):
+        b = sets[r % n_sets]
+        x, ids, g = dev[(r % n_sets) % n_mb]
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        ctx.dispatch(x, ids, b.counts, b.x_perm, b.slot_to_row, b.row_to_token, stream=stream)
+        e1.record(stream)
+        ctx.combine(b.y_perm, b.slot_to_row, g, b.out, stream=stream)
+        e2.record(stream)
+        torch.cuda.synchronize()
+        if r >= n_sets:                                           # the first round warms instruction caches only
+            t_disp.append(e0.elapsed_time(e1))
+            t_comb.append(e1.elapsed_time(e2))
+    ctx.check_status()
+    io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
+    del sets
+    torch.cuda.empty_cache()
+    return {"buffer_sets": n_sets, "footprint_mb": n_sets * per_set / 1e6,
+            "dispatch_us": float(np.median(t_disp)) * 1e3, "combine_us": float(np.median(t_comb)) * 1e3,
+            "dispatch_gbs_cold": io_bytes / (float(np.median(t_disp)) * 1e-3) / 1e9,
+            "combine_gbs_cold": io_bytes / (float(np.median(t_comb)) * 1e-3) / 1e9,
+            "note": "stand-alone feplb_dispatch (histogram, scan, ranking, gather) and feplb_combine, one call per "
+                    "buffer set in rotation; the in-pipeline (warm) figures are roofline.dispatch_gbs / combine_gbs"}
+
+
+def pick_bf16_peak(peaks, clocks):
+    """The bf16 denominator that matches the clock regime of the run it divides: the burst figure
+    when the SM clock sat within 5 % of its maximum and no power cap was active, else the sustained one."""
+    sus = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
+    if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        burst = clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"] and "sw_power_cap" not in clocks.get("reasons", [])
+        return (peaks["bf16_tflops"], "burst") if burst else (sus, "sustained")
+    return sus, "sustained (no clock samples)"
+
+
+def merged_timeline(st):
+    """One forward on one time axis, [name, start_us, end_us], origin = the forward's first kernel.
+    Device intervals come from CUDA events; the host marks of the planner thread are placed
+    relative to the instant the counts left the device (the thread polls pinned memory, so it sees
+    them within a PCIe write of the scan kernel's end)."""
+    if not st or not st.get("dev_total_us"):
+        return None
+    counts_at = st["dev_hist_us"]
+    h0 = st["host_counts_ready_us"]
+    s0 = counts_at + st["dev_counts_to_static_start_us"]
+    s1 = counts_at + st["dev_counts_to_static_end_us"]
+    d1 = st["dev_total_us"] - st["dev_combine_us"]
+    tl = [["hist+scan (counts to host)", 0.0, counts_at],
+          ["rank+gather (dispatch)", counts_at, counts_at + st["dev_dispatch_us"]],
+          ["static FFN (pass 1 + pass 2)", s0, s1],
+          ["host: counts seen by planner", counts_at, counts_at],
+          ["host: greedy plan", counts_at + st["host_plan_done_us"] - h0 - st["plan_us"], counts_at + st["host_plan_done_us"] - h0],
+          ["host: table upload enqueued", counts_at + st["host_upload_enqueued_us"] - h0, counts_at + st["host_upload_enqueued_us"] - h0],
+          ["dynamic FFN (pass 1 + pass 2)", d1 - st["dev_dynamic_ffn_us"], d1],
+          ["combine", d1, st["dev_total_us"]]]
+    if st.get("phase2_copy_bytes"):
+        tl.insert(6, ["phase-2 weight copies (copy engines)", counts_at + st["host_upload_enqueued_us"] - h0,
+                      counts_at + st["dev_counts_to_copies_done_us"]])
+    return [[n, round(a, 2), round(b, 2)] for n, a, b in tl]
 
 
 def run_sweep(args):
@@ -480,40 +588,75 @@ def _time_e2e(args, w, ctx, buf, host, d_w1, d_w3, d_w2, stream, barrier, world,
     return whole_job_throughput(world, args.steps, w.T, max_over_ranks(e2e_ms, world, "cuda"))
 
 
+def time_oracle_single_thread(w, sample_tokens, weights):
+    """The oracle with its BLAS limited to one thread (the plain loops are single-threaded anyway)."""
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return None
+    with threadpool_limits(limits=1):
+        val, _, n_tok = time_oracle(w, 1, 0, sample_tokens, weights)
+    return {"value": val, "sample_tokens": n_tok}
+
+
 def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals, n_fw, e2e_value, h2d, d2h, strag, weights, n_mb):
     if rank == 0:
         peaks = _peaks()
         ffn_us = totals["dev_static_ffn_us"] + totals["dev_dynamic_ffn_us"]
-        gemm_launches = 4 * n_fw
-        flops_launch = gemm_flops(w) / 4.0
+        per_fw = FFN_LAUNCHES_PER_FORWARD
+        gemm_launches = per_fw * n_fw
+        flops_launch = gemm_flops(w) / per_fw
         achieved = (flops_launch / (ffn_us * 1e-6 / gemm_launches)) / 1e12 if ffn_us > 0 else None
-        # a kernel timed inside a long step: the sustained bf16 figure is the honest denominator
-        peak = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
+        # the denominator follows the clock regime of the pass the kernel times were taken in
+        clk2 = getattr(args, "clocks_stage_pass", None)
+        peak, regime = pick_bf16_peak(peaks, clk2)
+        sus = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
         io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
+        cold = getattr(args, "cold", None) or {}
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
         roof = {"bound": "tensor", "kernel": "k_grouped_gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak if achieved else None, "peak_source": peaks["source"] + " (sustained)",
+                "frac": achieved / peak if achieved else None,
+                "peak_source": f"{peaks['source']} ({regime}: chosen from the SM clock and power-cap state sampled during this pass)",
+                "clocks": clk2,
                 "frac_of_burst": achieved / peaks["bf16_tflops"] if achieved else None,
+                "frac_of_sustained": achieved / sus if achieved else None,
                 "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name),
+                "traffic": traffic["bytes"] if traffic else None, "traffic_source": traffic["source"] if traffic else None,
                 "launches_timed": gemm_launches, "avg_launch_us": ffn_us / gemm_launches if gemm_launches else None,
                 "dispatch_gbs": io_bytes / (totals["dev_dispatch_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_dispatch_us"] else None,
                 "combine_gbs": io_bytes / (totals["dev_combine_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_combine_us"] else None,
+                "dispatch_gbs_cold": cold.get("dispatch_gbs_cold"), "combine_gbs_cold": cold.get("combine_gbs_cold"),
                 "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_nominal_gbs": 7700.0}
         stage_us = {k: (v / n_fw if n_fw else None) for k, v in totals.items()}
+        # the targets the task statement sets for config 2, as this run meets them or not
+        targets = None
+        if achieved:
+            hbm = peaks["hbm_gbs"]
+            targets = {"gemm_ge_0.60_of_burst_bf16_peak": bool(achieved / peaks["bf16_tflops"] >= 0.60),
+                       "dispatch_ge_0.60_of_hbm_peak": bool(roof["dispatch_gbs"] and roof["dispatch_gbs"] / hbm >= 0.60),
+                       "combine_ge_0.60_of_hbm_peak": bool(roof["combine_gbs"] and roof["combine_gbs"] / hbm >= 0.60),
+                       "dispatch_cold_ge_0.60_of_hbm_peak": bool(cold.get("dispatch_gbs_cold", 0) / hbm >= 0.60) if cold else None,
+                       "combine_cold_ge_0.60_of_hbm_peak": bool(cold.get("combine_gbs_cold", 0) / hbm >= 0.60) if cold else None}
         # CPU oracle on the host cores: a bounded sample of the same workload
         cpu = None
         if not args.quick:
             cpu_val, cpu_ms, n_tok = time_oracle(w, 2, 1, min(w.T, 4096), weights)
             cpu = {"value": cpu_val, "unit": UNIT, "cores": _oracle_threads(), "kind": "oracle",
-                   "sample": f"first {n_tok} tokens of 2 micro-batches, whole path (numpy fp64 oracle)"}
+                   "sample": f"first {n_tok} tokens of 2 micro-batches, whole path (numpy fp64 oracle)",
+                   "single_thread": time_oracle_single_thread(w, min(w.T, 512), weights)}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": _config_dict(w, args),
+            "repeats": getattr(args, "repeats", 1),
+            "block_ms": {"median": ms_total, "min": getattr(args, "block_ms_min", None), "max": getattr(args, "block_ms_max", None),
+                         "note": "each block is exactly `steps` steps between barrier + synchronize; blocks repeat until "
+                                 f"{args.min_timed_ms:.0f} ms are timed; value and ms_per_step are the median block's"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": int(launches), "clocks": clocks, "roofline": roof,
-            "cpu_baseline": cpu, "stage_us": stage_us, "straggler": strag,
-            # stage_us and roofline come from a second pass of the same K steps with per-stage
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "targets_cfg2": targets if w.name == "cfg2" else None,
+            "cpu_baseline": cpu, "stage_us": stage_us, "timeline": merged_timeline(stage_us), "cold_io": cold or None,
+            "straggler": strag,
+            # stage_us, timeline and roofline come from a second pass of the same blocks with per-stage
             # events on; those events cost time, so that pass is slower than ms_per_step
             "ms_per_step_with_stage_events": getattr(args, "ms_instrumented", None),
         }
@@ -592,6 +735,9 @@ def main():
     ap.add_argument("--backward", action="store_true", help="also time forward + backward (weight gradients included)")
     ap.add_argument("--phase2", action="store_true",
                     help="really copy migrated experts' weights into the receive buffer (copy engines) during the static GEMM")
+    ap.add_argument("--min-timed-ms", type=float, default=1000.0,
+                    help="repeat the block of --steps steps until this much device time has been timed (median block reported)")
+    ap.add_argument("--max-repeats", type=int, default=400)
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,
@@ -599,6 +745,8 @@ def main():
     ap.add_argument("--sensitivity", action="store_true",
                     help="host-only table: straggler reduction vs dyn, policy, mask, split (no GPU)")
     args = ap.parse_args()
+    if args.quick and args.min_timed_ms == 1000.0:
+        args.min_timed_ms = 0.0                     # profiling runs: one block per pass, few launches
     if args.sensitivity:
         run_sensitivity(args)
         return
