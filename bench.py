@@ -34,7 +34,6 @@ UNIT = "tokens/s"
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     "cfg2": {"bytes": 190.0e6, "source": "profiles/k_grouped_gemm_cfg2.md: 760 MB over the 4 launches of one forward"},
 }
-FFN_LAUNCHES_PER_FORWARD = 4    # static pass 1 / pass 2, dynamic pass 1 / pass 2
 
 
 def _peaks():
@@ -227,6 +226,7 @@ def run_cuda(args, w):
     B.build()
     cfg = F.config_from_workload(w, phase2_copy=1 if args.phase2 else 0, split=1 if args.split else 0)
     ctx = F.Context(cfg)
+    ctx.set_gemm_form({"auto": F.FORM_AUTO, "single": F.FORM_SINGLE, "pair": F.FORM_PAIR, "weight_m": F.FORM_WEIGHT_M}[args.form])
     buf = F.Buffers(cfg)
 
     weights = W.gen_weights(w)
@@ -382,16 +382,28 @@ def merged_timeline(st):
     s0 = counts_at + st["dev_counts_to_static_start_us"]
     s1 = counts_at + st["dev_counts_to_static_end_us"]
     d1 = st["dev_total_us"] - st["dev_combine_us"]
+    host = [["host: counts seen by planner", counts_at, counts_at],
+            ["host: greedy plan", counts_at + st["host_plan_done_us"] - h0 - st["plan_us"], counts_at + st["host_plan_done_us"] - h0],
+            ["host: dynamic table published / upload enqueued", counts_at + st["host_upload_enqueued_us"] - h0,
+             counts_at + st["host_upload_enqueued_us"] - h0]]
+    if st.get("ffn_launches", 4) < 3:
+        # weights-on-M form: one launch per pass; the marks inside the launches come from the GPU's timer
+        p1e = s0 + st["dev_ffn_pass1_us"]
+        tl = [["hist+scan (counts to host)", 0.0, counts_at],
+              ["rank+gather (dispatch)", counts_at, counts_at + st["dev_dispatch_us"]],
+              ["FFN pass 1: static groups (until the first CTA runs out of them)", s0, s1]] + host + [
+              ["FFN pass 1: remaining static and dynamic groups", s1, p1e],
+              ["FFN pass 2: static, then dynamic groups", d1 - st["dev_ffn_pass2_us"], d1],
+              ["longest device-side wait for the dynamic table", s1, s1 + st["dev_plan_wait_us"]],
+              ["combine", d1, st["dev_total_us"]]]
+        return [[n, round(a, 2), round(b, 2)] for n, a, b in tl]
     tl = [["hist+scan (counts to host)", 0.0, counts_at],
           ["rank+gather (dispatch)", counts_at, counts_at + st["dev_dispatch_us"]],
-          ["static FFN (pass 1 + pass 2)", s0, s1],
-          ["host: counts seen by planner", counts_at, counts_at],
-          ["host: greedy plan", counts_at + st["host_plan_done_us"] - h0 - st["plan_us"], counts_at + st["host_plan_done_us"] - h0],
-          ["host: table upload enqueued", counts_at + st["host_upload_enqueued_us"] - h0, counts_at + st["host_upload_enqueued_us"] - h0],
+          ["static FFN (pass 1 + pass 2)", s0, s1]] + host + [
           ["dynamic FFN (pass 1 + pass 2)", d1 - st["dev_dynamic_ffn_us"], d1],
           ["combine", d1, st["dev_total_us"]]]
     if st.get("phase2_copy_bytes"):
-        tl.insert(6, ["phase-2 weight copies (copy engines)", counts_at + st["host_upload_enqueued_us"] - h0,
+        tl.insert(6, ["phase-2 weight copies", counts_at + st["host_upload_enqueued_us"] - h0,
                       counts_at + st["dev_counts_to_copies_done_us"]])
     return [[n, round(a, 2), round(b, 2)] for n, a, b in tl]
 
@@ -603,7 +615,7 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
     if rank == 0:
         peaks = _peaks()
         ffn_us = totals["dev_static_ffn_us"] + totals["dev_dynamic_ffn_us"]
-        per_fw = FFN_LAUNCHES_PER_FORWARD
+        per_fw = int(round(totals.get("ffn_launches", 0) / n_fw)) if n_fw and totals.get("ffn_launches") else 4
         gemm_launches = per_fw * n_fw
         flops_launch = gemm_flops(w) / per_fw
         achieved = (flops_launch / (ffn_us * 1e-6 / gemm_launches)) / 1e12 if ffn_us > 0 else None
@@ -614,7 +626,8 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
         io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
         cold = getattr(args, "cold", None) or {}
         traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
-        roof = {"bound": "tensor", "kernel": "k_grouped_gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+        roof = {"bound": "tensor", "kernel": "k_ffn_wm (weights on M, static + dynamic groups per launch)" if per_fw == 2 else "k_grouped_gemm",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak if achieved else None,
                 "peak_source": f"{peaks['source']} ({regime}: chosen from the SM clock and power-cap state sampled during this pass)",
                 "clocks": clk2,
@@ -738,6 +751,8 @@ def main():
     ap.add_argument("--min-timed-ms", type=float, default=1000.0,
                     help="repeat the block of --steps steps until this much device time has been timed (median block reported)")
     ap.add_argument("--max-repeats", type=int, default=400)
+    ap.add_argument("--form", default="auto", choices=["auto", "single", "pair", "weight_m"],
+                    help="grouped-GEMM form of the forward launches (feplb_set_gemm_form); auto is the library's choice")
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,

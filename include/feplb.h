@@ -46,7 +46,7 @@ typedef enum {
   FEPLB_E_RANGE = -2,   /* an expert id outside [0, E) was seen on the device */
   FEPLB_E_CUDA = -3,    /* a CUDA runtime/driver call failed; text in feplb_last_error */
   FEPLB_E_NOMEM = -4,   /* an allocation failed, or a caller-sized array is too small */
-  FEPLB_E_TIMEOUT = -5, /* a bounded host wait expired */
+  FEPLB_E_TIMEOUT = -5, /* a bounded host wait expired, or the GEMM's bounded wait for the plan did */
   FEPLB_E_STATE = -6,   /* call order violated (e.g. plan_wait without plan_async) */
   FEPLB_E_DEVICE = -7   /* a bounded device-side wait gave up, or counts disagree with ids */
 } feplb_status;
@@ -54,7 +54,7 @@ typedef enum {
 enum { FEPLB_POLICY_LITERAL = 0, FEPLB_POLICY_FIRST_FIT = 1 };
 enum { FEPLB_MASK_GIVEN = 0, FEPLB_MASK_REACTIVE = 1 };
 enum { FEPLB_FFN_ALL = 0, FEPLB_FFN_STATIC = 1, FEPLB_FFN_DYNAMIC = 2 };
-enum { FEPLB_FORM_AUTO = -1, FEPLB_FORM_SINGLE = 0, FEPLB_FORM_PAIR = 1 };
+enum { FEPLB_FORM_AUTO = -1, FEPLB_FORM_SINGLE = 0, FEPLB_FORM_PAIR = 1, FEPLB_FORM_WEIGHT_M = 2 };
 
 /* Layer geometry and balancer parameters.
  * Requirements: E % R == 0; d % 128 == 0; f % 64 == 0; 1 <= K <= 32; E <= 1024;
@@ -114,6 +114,13 @@ typedef struct {
   double dev_total_us;
   double dev_counts_to_copies_done_us;  /* device: counts copied -> Phase-2 weight copies landed (0 if none) */
   double phase2_copy_bytes;             /* bytes moved by those copies */
+  /* Weights-on-M form only (one launch per pass walks the static, then the dynamic groups); the
+   * marks are taken inside the kernels from the GPU's global timer.  There dev_static_ffn_us is the
+   * whole expert FFN, dev_dynamic_ffn_us is 0, dev_counts_to_static_start_us ends at the first CTA's
+   * start and dev_counts_to_static_end_us at the first moment a CTA ran out of static work. */
+  double dev_ffn_pass1_us, dev_ffn_pass2_us; /* device: first CTA's start -> last CTA's end of each pass */
+  double dev_plan_wait_us;              /* device: longest time a CTA spent waiting for the dynamic table */
+  double ffn_launches;                  /* GEMM launches of the forward: 4 (static, dynamic x 2 passes) or 2 */
 } feplb_timeline;
 
 typedef struct feplb_ctx feplb_ctx;
@@ -382,12 +389,23 @@ int feplb_timeline_totals(feplb_ctx* ctx, feplb_timeline* sum, int64_t* n_forwar
  * the context stays usable.  Not allowed while a plan is pending. */
 int feplb_set_planner_timeout(feplb_ctx* ctx, int32_t timeout_ms);
 /* Which form of the grouped-GEMM kernel the context uses.  forward_form: FEPLB_FORM_AUTO (default:
- * chosen per group table from the rows per group), FEPLB_FORM_SINGLE (one CTA per 128-row tile) or
- * FEPLB_FORM_PAIR (clusters of two CTAs on 256-row tiles) for every forward launch.
+ * chosen from the geometry and, per group table, from the rows per group), FEPLB_FORM_SINGLE (one
+ * CTA per 128-row tile), FEPLB_FORM_PAIR (clusters of two CTAs on 256-row tiles) or
+ * FEPLB_FORM_WEIGHT_M (weight tiles on the M side, up to 256 rows of a group on the N side; in
+ * feplb_moe_forward one launch per pass then runs the static groups and, after picking the
+ * planner's table up on the device, the dynamic groups; needs f % 128 == 0, d % 256 == 0 and
+ * 2*E + R*max_num_dyn <= 1024, else FEPLB_E_INVALID) for every forward launch.
  * backward_pair: -1 (default: chosen from the geometry) or a mask, bit 0 = activation-gradient
  * GEMMs in the pair form, bit 1 = weight-gradient GEMMs in the pair form.  Results do not depend
  * on the form beyond fp32 summation order.  Not allowed while a plan is pending. */
 int feplb_set_gemm_form(feplb_ctx* ctx, int32_t forward_form, int32_t backward_pair);
+/* Test and tuning aid for the weights-on-M form of feplb_moe_forward.  planner_delay_us: the
+ * planner thread sleeps that long before it publishes its table (0 = off), so that the GEMM's
+ * device-side wait for the table really is entered.  device_wait_limit_us: bound of that wait
+ * (0 = the default, 400 ms); when it expires the kernels skip the dynamic groups, raise a status
+ * bit that feplb_check_status reports as FEPLB_E_TIMEOUT, and return normally.  Not allowed while
+ * a plan is pending. */
+int feplb_set_planner_timing(feplb_ctx* ctx, int32_t planner_delay_us, int32_t device_wait_limit_us);
 /* Self-test of the device-side bounded waits: launches one thread that waits, with the routine
  * the GEMM kernels use, on an mbarrier nothing ever completes, limited to limit_us microseconds.
  * Returns FEPLB_OK if the wait gave up, raised the status bit and the kernel returned normally;

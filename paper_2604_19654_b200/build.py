@@ -17,7 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfeplb.so")
 SOURCES = ["feplb_plan.cpp", "feplb_api.cu", "feplb_route.cu", "feplb_combine.cu", "feplb_gemm.cu",
-           "feplb_noalloc.cu", "feplb_gemm_bwd.cu"]
+           "feplb_noalloc.cu", "feplb_gemm_bwd.cu", "feplb_gemm_wm.cu"]
 
 
 def _nvcc() -> str:

@@ -27,6 +27,7 @@ inline double us_since(clk::time_point t0) {
 enum JobState { JOB_IDLE = 0, JOB_PENDING = 1, JOB_RUNNING = 2, JOB_DONE = 3 };
 enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_COPIES, EV_N };
 constexpr int kEvRing = 16;   // forwards whose stage events may be outstanding
+constexpr int kStampWords = 16;   // [0..3] pass 1, [4..7] pass 2 (see WmParams::stamps), [8] counts left the device
 }  // namespace
 
 struct feplb_ctx {
@@ -40,6 +41,21 @@ struct feplb_ctx {
   int gemm_pair_forced = -1;   // feplb_set_gemm_form: 0/1 forces one form everywhere, -1 = chosen per table
   int bwd_pair = 0;            // backward GEMMs in the pair form: bit 0 activation gradients, bit 1 weight gradients
   int gemm_pair_auto = 0, bwd_pair_auto = 0;   // the choices feplb_create derived from the geometry
+  bool wm_ok = false;          // the weights-on-M form supports this geometry
+  bool wm = false;             // ... and is the form in use (feplb_create's choice or feplb_set_gemm_form)
+  bool wm_auto = false;
+  int32_t planner_delay_us = 0;        // test aid: the planner sleeps before it publishes its table
+  int32_t device_wait_limit_us = 0;    // bound of the GEMM's wait for the table (0: default)
+  // weights-on-M form: the words through which a running GEMM launch learns that the dynamic table exists
+  int32_t* h_dyn_tab32 = nullptr;                    // pinned + mapped: the dynamic table as 32-byte entries tagged with the sequence number
+  int32_t* h_dyn_tab32_dev = nullptr;                // its device address
+  int32_t* d_dyn_tab32 = nullptr;                    // device copy, made by the GEMM's claiming CTA
+  unsigned long long* d_dyn_ready = nullptr;         // device words: [0] ready, [1] claim
+  unsigned long long* h_dyn_ready = nullptr;         // pinned + mapped word, set by the planner thread
+  unsigned long long* h_dyn_ready_dev = nullptr;     // its device address
+  unsigned long long* d_stamps = nullptr;            // [kEvRing][kStampWords] globaltimer marks of the kernels
+  unsigned long long* h_stamps = nullptr;            // pinned copy, filled at the end of a timed forward
+  bool job_wm = false;
 
   // device scratch
   int32_t* d_block_hist = nullptr;
@@ -210,18 +226,44 @@ void planner_main(feplb_ctx* c) {
             if (i < c->plan.n_moves) gr.is_dynamic = 2 + move_slot[i];
           }
           if (ce == cudaSuccess && c->copy_bytes > 0) ce = cudaEventRecord(c->ev[EV_COPIES], c->copy_stream);
+          if (ce != cudaSuccess) c->copy_bytes = 0;
           c->tl.phase2_copy_bytes = c->copy_bytes;
         }
         if (ce != cudaSuccess) rc = FEPLB_E_CUDA;
         int64_t dyn_rows = 0;
         for (int i = 0; i < n; ++i) dyn_rows += c->h_dyn_groups[i].rows;
-        c->dyn_pair = c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (n > 0 && dyn_rows >= (int64_t)512 * n);
+        c->dyn_pair = c->gemm_pair_forced >= 0 ? c->gemm_pair_forced == FEPLB_FORM_PAIR : (n > 0 && dyn_rows >= (int64_t)512 * n);
         cudaError_t e = cudaSuccess;
-        if (n) e = feplb_launch_upload_groups(c->h_dyn_groups_dev, c->d_dyn_groups, n, c->copy_stream);
-        if (e == cudaSuccess) e = cudaEventRecord(c->ev_plan, c->copy_stream);
+        if (c->job_wm) {
+          // A GEMM launch may already be running and waiting for this table (the merged launches
+          // are never combined with Phase-2 copies): publish it from here, with a plain store into
+          // mapped host memory, so that the waiting kernel depends on this thread alone.  The first
+          // CTA that sees the word brings the table into device memory for the others; there is no
+          // upload kernel on this path (it could not be relied on to run beside a kernel that holds
+          // every SM, and a late one would overwrite the next forward's table).
+          if (c->planner_delay_us > 0) std::this_thread::sleep_for(std::chrono::microseconds(c->planner_delay_us));
+          const unsigned long long word = ((unsigned long long)(uint32_t)c->job_flag_seq << 32) | (uint32_t)n;
+          for (int i = 0; i < n; ++i) {
+            const feplb_group& gr = c->h_dyn_groups[i];
+            volatile int32_t* t = c->h_dyn_tab32 + 8 * i;
+            t[0] = gr.expert; t[1] = gr.row_start; t[2] = gr.rows; t[3] = gr.exec_rank;
+            t[4] = gr.is_dynamic; t[5] = c->job_flag_seq; t[6] = 0; t[7] = 0;
+          }
+          std::atomic_thread_fence(std::memory_order_release);
+          *(volatile unsigned long long*)c->h_dyn_ready = word;
+          c->tl.host_upload_enqueued_us = us_since(c->t0);
+        } else {
+          if (n) e = feplb_launch_upload_groups(c->h_dyn_groups_dev, c->d_dyn_groups, n, c->copy_stream);
+          if (e == cudaSuccess) e = cudaEventRecord(c->ev_plan, c->copy_stream);
+          c->tl.host_upload_enqueued_us = us_since(c->t0);
+        }
         if (e != cudaSuccess) rc = FEPLB_E_CUDA;
       }
-      c->tl.host_upload_enqueued_us = us_since(c->t0);
+    }
+    if (rc != FEPLB_OK && c->job_wm && c->job_flag_seq) {
+      // the launches of this forward must not wait for a table that will not come: an empty one
+      std::atomic_thread_fence(std::memory_order_release);
+      *(volatile unsigned long long*)c->h_dyn_ready = (unsigned long long)(uint32_t)c->job_flag_seq << 32;
     }
     {
       std::lock_guard<std::mutex> lk(c->mu);
@@ -281,7 +323,24 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   c->nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   const int cap_moves = cfg->R * cfg->max_num_dyn;
   const int cap_groups = cfg->E + cap_moves;
+  // Weights-on-M form: pays while groups are a few hundred rows (less padding, an expert's weights cross
+  // the L2 port once per 256 rows); from ~1000 rows per expert the two-CTA form keeps its lead because
+  // it can overlap every tile's epilogue with the next tile's MMAs.
+  c->wm_ok = feplb_wm_supported(cfg->E, cfg->d, cfg->f, cfg->E + cap_groups);
+  c->wm_auto = c->wm = c->wm_ok && S < (int64_t)FEPLB_WM_AUTO_ROWS_PER_EXPERT * cfg->E;
   bool ok = true;
+  ok = ok && cudaMalloc(&c->d_dyn_ready, 2 * sizeof(unsigned long long)) == cudaSuccess &&     // [0] ready word, [1] claim word
+       cudaMemset(c->d_dyn_ready, 0, 2 * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaHostAlloc(&c->h_dyn_ready, sizeof(unsigned long long), cudaHostAllocMapped) == cudaSuccess &&
+       cudaHostGetDevicePointer(&c->h_dyn_ready_dev, c->h_dyn_ready, 0) == cudaSuccess;
+  if (ok) *c->h_dyn_ready = 0;
+  ok = ok && cudaHostAlloc(&c->h_dyn_tab32, 32 * (size_t)(cap_groups > 0 ? cap_groups : 1), cudaHostAllocMapped) == cudaSuccess &&
+       cudaHostGetDevicePointer(&c->h_dyn_tab32_dev, c->h_dyn_tab32, 0) == cudaSuccess;
+  if (ok) memset(c->h_dyn_tab32, 0, 32 * (size_t)(cap_groups > 0 ? cap_groups : 1));
+  ok = ok && cudaMalloc(&c->d_dyn_tab32, 32 * (size_t)(cap_groups > 0 ? cap_groups : 1)) == cudaSuccess &&
+       cudaMemset(c->d_dyn_tab32, 0, 32 * (size_t)(cap_groups > 0 ? cap_groups : 1)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_stamps, sizeof(unsigned long long) * kEvRing * kStampWords) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->h_stamps, sizeof(unsigned long long) * kEvRing * kStampWords) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_block_hist, sizeof(int32_t) * (size_t)(c->nb > 0 ? c->nb : 1) * cfg->E) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_pad_off, sizeof(int32_t) * (cfg->E + 1)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(uint32_t)) == cudaSuccess;
@@ -356,6 +415,12 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFree(c->d_recv_w1);
   cudaFree(c->d_recv_w3);
   cudaFree(c->d_recv_w2);
+  cudaFree(c->d_dyn_ready);
+  cudaFree(c->d_dyn_tab32);
+  cudaFreeHost(c->h_dyn_tab32);
+  cudaFree(c->d_stamps);
+  cudaFreeHost(c->h_dyn_ready);
+  cudaFreeHost(c->h_stamps);
   cudaFreeHost(c->h_counts);
   cudaFreeHost(c->h_dyn_groups);
   cudaFreeHost(c->h_status);
@@ -391,6 +456,8 @@ extern "C" int feplb_check_status(feplb_ctx* c, void* stream) {
   CUDA_TRY(c, cudaStreamSynchronize(st));
   const uint32_t s = *c->h_status;
   if (s & FEPLB_ST_WAIT) return fail(c, FEPLB_E_DEVICE, "a bounded device-side wait gave up (status 0x%x)", s);
+  if (s & FEPLB_ST_PLAN)
+    return fail(c, FEPLB_E_TIMEOUT, "the expert GEMM gave up waiting for the planner's dynamic group table (status 0x%x)", s);
   if (s & FEPLB_ST_GROUP) return fail(c, FEPLB_E_DEVICE, "malformed group entry (status 0x%x)", s);
   if (s & FEPLB_ST_COUNTS) return fail(c, FEPLB_E_DEVICE, "counts disagree with topk_ids (status 0x%x)", s);
   if (s & FEPLB_ST_RANGE) return fail(c, FEPLB_E_RANGE, "expert id outside [0, E) (status 0x%x)", s);
@@ -440,14 +507,15 @@ extern "C" int feplb_home_groups(feplb_ctx* c, const int32_t* counts, const uint
   return FEPLB_OK;
 }
 
+// `dyn` != nullptr: weights-on-M launches that go on to the planner's dynamic table after `groups`.
 static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void* w3, const void* w2,
                     const feplb_group* groups, int32_t n_groups, int32_t which, void* h, void* y, cudaStream_t st,
-                    int pair = -1) {
+                    int pair = -1, const feplb_wm_dyn* dyn = nullptr) {
   if (pair < 0) pair = c->gemm_pair_default;
   if (n_groups < 0 || n_groups > FEPLB_MAX_GROUPS) return fail(c, FEPLB_E_INVALID, "expert_ffn: n_groups out of range");
   if (which != FEPLB_FFN_ALL && which != FEPLB_FFN_STATIC && which != FEPLB_FFN_DYNAMIC)
     return fail(c, FEPLB_E_INVALID, "expert_ffn: bad selector");
-  if (n_groups == 0 || c->s_cap == 0) return FEPLB_OK;
+  if ((n_groups == 0 && !dyn) || c->s_cap == 0) return FEPLB_OK;
   int rc = check_dev_ptrs(c, {x_perm, w1, w3, w2, h, y});
   if (rc != FEPLB_OK) return rc;
   if (!groups) return fail(c, FEPLB_E_INVALID, "expert_ffn: null group table");
@@ -458,6 +526,11 @@ static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void
   a.status = c->d_status; a.num_sms = c->num_sms; a.pair = pair;
   a.ab_out = c->d_preact;
   a.recv_w1 = c->d_recv_w1; a.recv_w3 = c->d_recv_w3; a.recv_w2 = c->d_recv_w2; a.n_recv_slots = c->n_recv_slots;
+  if (c->wm && n_groups + (dyn ? dyn->max_groups : 0) <= FEPLB_WM_MAX_ENTRIES) {
+    const feplb_wm_dyn none;
+    return feplb_launch_expert_ffn_wm(a, dyn ? *dyn : none, st, &c->launches, c->err, sizeof(c->err));
+  }
+  if (dyn) return fail(c, FEPLB_E_STATE, "expert_ffn: merged launch without the weights-on-M form");
   return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err));
 }
 
@@ -497,6 +570,7 @@ extern "C" int feplb_plan_async(feplb_ctx* c, const int32_t* counts, const uint8
     std::lock_guard<std::mutex> lk(c->mu);
     c->job_mask = dyn_mask_host;
     c->job_flag_seq = 0;
+    c->job_wm = false;
     c->job = JOB_PENDING;
   }
   c->cv.notify_all();
@@ -504,11 +578,12 @@ extern "C" int feplb_plan_async(feplb_ctx* c, const int32_t* counts, const uint8
 }
 
 // Whole-layer path: the counts of this forward arrive in h_counts with sequence number `seq`.
-static int plan_kick_flag(feplb_ctx* c, const uint8_t* dyn_mask_host, int32_t seq) {
+static int plan_kick_flag(feplb_ctx* c, const uint8_t* dyn_mask_host, int32_t seq, bool wm) {
   {
     std::lock_guard<std::mutex> lk(c->mu);
     if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "moe_forward: a plan is already pending");
     c->job_mask = dyn_mask_host;
+    c->job_wm = wm;
     c->job_flag_seq = seq;
     c->job = JOB_PENDING;
   }
@@ -516,9 +591,8 @@ static int plan_kick_flag(feplb_ctx* c, const uint8_t* dyn_mask_host, int32_t se
   return FEPLB_OK;
 }
 
-extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out* plan_copy,
-                               const feplb_group** dyn_groups_dev, int32_t* n_dyn_groups, void* stream) {
-  if (!c) return FEPLB_E_INVALID;
+// Waits for the planner's job and returns the context to idle; copies the plan out.
+static int join_planner(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out* plan_copy) {
   int rc;
   {
     std::unique_lock<std::mutex> lk(c->mu);
@@ -540,9 +614,17 @@ extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out*
     memcpy(plan_copy->load_before, c->plan.load_before, sizeof(int64_t) * c->cfg.R);
     memcpy(plan_copy->load_after, c->plan.load_after, sizeof(int64_t) * c->cfg.R);
   }
+  if (c->n_dyn_groups > 0 && !c->job_wm) ++c->launches;     // the planner thread's table upload kernel
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_plan_wait(feplb_ctx* c, int32_t timeout_ms, feplb_plan_out* plan_copy,
+                               const feplb_group** dyn_groups_dev, int32_t* n_dyn_groups, void* stream) {
+  if (!c) return FEPLB_E_INVALID;
+  int rc = join_planner(c, timeout_ms, plan_copy);
+  if (rc != FEPLB_OK) return rc;
   if (dyn_groups_dev) *dyn_groups_dev = c->d_dyn_groups;
   if (n_dyn_groups) *n_dyn_groups = c->n_dyn_groups;
-  if (c->n_dyn_groups > 0) ++c->launches;      // the planner thread's table upload kernel
   CUDA_TRY(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_plan, 0));
   return FEPLB_OK;
 }
@@ -564,6 +646,20 @@ static int harvest_slot(feplb_ctx* c, int r) {
   t.dev_counts_to_static_end_us = el(ev[EV_COUNTS], ev[EV_STATIC1]);
   t.dev_total_us = el(ev[EV_T0], ev[EV_COMBINE]);
   t.dev_counts_to_copies_done_us = t.phase2_copy_bytes > 0 ? el(ev[EV_COUNTS], ev[EV_COPIES]) : 0.0;
+  if (t.ffn_launches == 2) {
+    // weights-on-M form: marks taken inside the kernels (all ones = never written)
+    const unsigned long long* sp = c->h_stamps + (size_t)r * kStampWords;
+    const unsigned long long none = ~0ull;
+    auto span = [&](unsigned long long a, unsigned long long b) { return a != none && b != none && b >= a ? (b - a) * 1e-3 : 0.0; };
+    const unsigned long long t_counts = sp[8], p1_start = sp[0], p1_first_dyn = sp[1], p1_end = sp[2] == none ? none : ~sp[2];
+    const unsigned long long p2_start = sp[4], p2_end = sp[6] == none ? none : ~sp[6];
+    t.dev_ffn_pass1_us = span(p1_start, p1_end);
+    t.dev_ffn_pass2_us = span(p2_start, p2_end);
+    t.dev_counts_to_static_start_us = span(t_counts, p1_start);
+    t.dev_counts_to_static_end_us = span(t_counts, p1_first_dyn != none ? p1_first_dyn : p1_end);
+    const unsigned long long w1 = sp[3] == none ? 0 : ~sp[3], w2 = sp[7] == none ? 0 : ~sp[7];
+    t.dev_plan_wait_us = (w1 > w2 ? w1 : w2) * 1e-3;
+  }
   cudaGetLastError();
   const double* src = reinterpret_cast<const double*>(&t);
   double* dst = reinterpret_cast<double*>(&c->tl_sum);
@@ -605,6 +701,23 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   c->timeline_valid = true;
   c->tl.phase2_copy_bytes = 0;
   c->tl.dev_counts_to_copies_done_us = 0;
+  // Weights-on-M form: one launch per pass runs the static groups and then the dynamic ones, whose
+  // table it picks up on the device, so everything is enqueued before the planner is joined.
+  // Not with Phase-2 weight copies: the dynamic groups would then wait, inside a kernel that holds
+  // every SM, for device-to-device copies that the driver may carry out with kernels of its own;
+  // that case keeps the four-launch order (the dynamic launches follow the copies in stream order).
+  const bool wm = c->wm && !g.phase2_copy;
+  c->tl.ffn_launches = wm ? 2 : 4;
+  c->tl.dev_ffn_pass1_us = c->tl.dev_ffn_pass2_us = c->tl.dev_plan_wait_us = 0;
+  unsigned long long* stamps = nullptr;
+  if (wm && c->timeline_on) {
+    stamps = c->d_stamps + (size_t)c->ev_slot * kStampWords;
+    CUDA_TRY(c, cudaMemsetAsync(stamps, 0xFF, sizeof(unsigned long long) * kStampWords, st));
+#ifdef FEPLB_PROBE
+    CUDA_TRY(c, cudaMemsetAsync(stamps + 10, 0, 8, st));
+    CUDA_TRY(c, cudaMemsetAsync(stamps + 12, 0, 8, st));
+#endif
+  }
   TL_EVENT(EV_T0);
   // step 1: counts, rank loads, segment offsets and the home group table in two launches; the
   // planner thread starts as soon as the counts reach the host
@@ -624,10 +737,10 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   const int32_t seq = c->flag_seq;
   CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
                                        rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
-                                       (int64_t)c->s_cap, c->d_status, c->h_counts_tagged, seq, st,
-                                       &c->launches));
+                                       (int64_t)c->s_cap, c->d_status, c->h_counts_tagged, seq,
+                                       stamps ? stamps + 8 : nullptr, st, &c->launches));
   c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
-  if ((rc = plan_kick_flag(c, dyn_mask_host, seq)) != FEPLB_OK) return rc;
+  if ((rc = plan_kick_flag(c, dyn_mask_host, seq, wm)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);
   // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move
@@ -641,25 +754,58 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "dispatch launch: %s", cudaGetErrorString(e));
   }
   TL_EVENT(EV_DISPATCH);
-  // step 4: static experts on their home ranks, from the group table built on the device
   TL_EVENT(EV_STATIC0);
-  if (rc == FEPLB_OK)
-    rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st);
-  TL_EVENT(EV_STATIC1);
-  c->tl.host_enqueue_static_done_us = us_since(c->t0);
-  // join the planner (always, so that the context returns to idle), then step 5
-  const feplb_group* dyn_groups = nullptr;
-  int32_t n_dyn = 0;
-  int rc_join = feplb_plan_wait(c, c->planner_timeout_ms + 500, plan_copy, &dyn_groups, &n_dyn, stream);
-  c->tl.host_join_us = us_since(c->t0);
-  if (rc != FEPLB_OK) return rc;
-  if (rc_join != FEPLB_OK) return rc_join;
-  TL_EVENT(EV_DYN0);
-  if ((rc = ffn_impl(c, x_perm, w1, w3, w2, dyn_groups, n_dyn, FEPLB_FFN_ALL, h_scratch, y_perm, st, c->dyn_pair)) != FEPLB_OK) return rc;
-  TL_EVENT(EV_DYN1);
-  // step 6
-  if ((rc = feplb_combine(c, y_perm, slot_to_row, gates, out, stream)) != FEPLB_OK) return rc;
-  TL_EVENT(EV_COMBINE);
+  if (wm) {
+    // steps 4 + 5 in two launches: static groups from the table built on the device, then the dynamic
+    // groups as soon as the planner has published them (bounded wait inside the kernel)
+    feplb_wm_dyn dyn;
+    dyn.table_dev = c->d_dyn_tab32; dyn.table_host = c->h_dyn_tab32_dev;
+    dyn.ready_dev = c->d_dyn_ready; dyn.ready_host = c->h_dyn_ready_dev;
+    dyn.claim = reinterpret_cast<uint32_t*>(c->d_dyn_ready + 1);
+    dyn.seq = (uint32_t)seq; dyn.max_groups = c->plan.cap_groups; dyn.stamps = stamps;
+    dyn.wait_limit_ns = 1000ull * (unsigned long long)c->device_wait_limit_us;
+    if (rc == FEPLB_OK)
+      rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st, -1, &dyn);
+    TL_EVENT(EV_STATIC1);
+    c->tl.host_enqueue_static_done_us = us_since(c->t0);
+    TL_EVENT(EV_DYN0);
+    TL_EVENT(EV_DYN1);
+    int rc_comb = rc == FEPLB_OK ? feplb_combine(c, y_perm, slot_to_row, gates, out, stream) : FEPLB_OK;
+    if (stamps && rc == FEPLB_OK && rc_comb == FEPLB_OK) {
+      cudaError_t e = cudaMemcpyAsync(c->h_stamps + (size_t)c->ev_slot * kStampWords, stamps,
+                                      sizeof(unsigned long long) * kStampWords, cudaMemcpyDeviceToHost, st);
+      if (e != cudaSuccess) rc_comb = fail(c, FEPLB_E_CUDA, "timeline copy: %s", cudaGetErrorString(e));
+    }
+    if (c->timeline_on && rc == FEPLB_OK && rc_comb == FEPLB_OK) {
+      cudaError_t e = cudaEventRecord(c->ev[EV_COMBINE], st);
+      if (e != cudaSuccess) rc_comb = fail(c, FEPLB_E_CUDA, "event record: %s", cudaGetErrorString(e));
+    }
+    // join the planner (always, so that the context returns to idle): everything is already enqueued
+    int rc_join = join_planner(c, c->planner_timeout_ms + 500, plan_copy);
+    c->tl.host_join_us = us_since(c->t0);
+    if (rc != FEPLB_OK) return rc;
+    if (rc_comb != FEPLB_OK) return rc_comb;
+    if (rc_join != FEPLB_OK) return rc_join;
+  } else {
+    // step 4: static experts on their home ranks, from the group table built on the device
+    if (rc == FEPLB_OK)
+      rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st);
+    TL_EVENT(EV_STATIC1);
+    c->tl.host_enqueue_static_done_us = us_since(c->t0);
+    // join the planner (always, so that the context returns to idle), then step 5
+    const feplb_group* dyn_groups = nullptr;
+    int32_t n_dyn = 0;
+    int rc_join = feplb_plan_wait(c, c->planner_timeout_ms + 500, plan_copy, &dyn_groups, &n_dyn, stream);
+    c->tl.host_join_us = us_since(c->t0);
+    if (rc != FEPLB_OK) return rc;
+    if (rc_join != FEPLB_OK) return rc_join;
+    TL_EVENT(EV_DYN0);
+    if ((rc = ffn_impl(c, x_perm, w1, w3, w2, dyn_groups, n_dyn, FEPLB_FFN_ALL, h_scratch, y_perm, st, c->dyn_pair)) != FEPLB_OK) return rc;
+    TL_EVENT(EV_DYN1);
+    // step 6
+    if ((rc = feplb_combine(c, y_perm, slot_to_row, gates, out, stream)) != FEPLB_OK) return rc;
+    TL_EVENT(EV_COMBINE);
+  }
   c->tl.host_return_us = us_since(c->t0);
   if (c->timeline_on) {
     c->ev_host[c->ev_slot] = c->tl;
@@ -796,15 +942,35 @@ extern "C" int feplb_set_planner_timeout(feplb_ctx* c, int32_t timeout_ms) {
 
 extern "C" int feplb_set_gemm_form(feplb_ctx* c, int32_t forward_form, int32_t backward_pair) {
   if (!c) return FEPLB_E_INVALID;
-  if (forward_form < FEPLB_FORM_AUTO || forward_form > FEPLB_FORM_PAIR)
-    return fail(c, FEPLB_E_INVALID, "set_gemm_form: forward_form must be FEPLB_FORM_AUTO, _SINGLE or _PAIR");
+  if (forward_form < FEPLB_FORM_AUTO || forward_form > FEPLB_FORM_WEIGHT_M)
+    return fail(c, FEPLB_E_INVALID, "set_gemm_form: forward_form must be FEPLB_FORM_AUTO, _SINGLE, _PAIR or _WEIGHT_M");
+  if (forward_form == FEPLB_FORM_WEIGHT_M && !c->wm_ok)
+    return fail(c, FEPLB_E_INVALID, "set_gemm_form: the weights-on-M form needs f %% 128 == 0, d %% 256 == 0 and "
+                                    "2*E + R*max_num_dyn <= %d", FEPLB_WM_MAX_ENTRIES);
   if (backward_pair < -1 || backward_pair > 3)
     return fail(c, FEPLB_E_INVALID, "set_gemm_form: backward_pair must be -1 (auto) or a 2-bit mask");
   std::lock_guard<std::mutex> lk(c->mu);
   if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "set_gemm_form: a plan is pending");
-  c->gemm_pair_forced = forward_form;
-  c->gemm_pair_default = forward_form == FEPLB_FORM_AUTO ? c->gemm_pair_auto : forward_form;
+  c->wm = forward_form == FEPLB_FORM_AUTO ? c->wm_auto : forward_form == FEPLB_FORM_WEIGHT_M;
+  c->gemm_pair_forced = forward_form == FEPLB_FORM_SINGLE || forward_form == FEPLB_FORM_PAIR ? forward_form : -1;
+  c->gemm_pair_default = c->gemm_pair_forced < 0 ? c->gemm_pair_auto : forward_form;
   c->bwd_pair = backward_pair < 0 ? c->bwd_pair_auto : backward_pair;
+  return FEPLB_OK;
+}
+
+#ifdef FEPLB_PROBE
+extern "C" int feplb_probe_stamps(feplb_ctx* c, unsigned long long* out) {
+  for (int i = 0; i < kStampWords; ++i) out[i] = c->h_stamps[(size_t)c->ev_slot * kStampWords + i];
+  return 0;
+}
+#endif
+
+extern "C" int feplb_set_planner_timing(feplb_ctx* c, int32_t planner_delay_us, int32_t device_wait_limit_us) {
+  if (!c || planner_delay_us < 0 || planner_delay_us > 1000000 || device_wait_limit_us < 0) return FEPLB_E_INVALID;
+  std::lock_guard<std::mutex> lk(c->mu);
+  if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "set_planner_timing: a plan is pending");
+  c->planner_delay_us = planner_delay_us;
+  c->device_wait_limit_us = device_wait_limit_us;
   return FEPLB_OK;
 }
 

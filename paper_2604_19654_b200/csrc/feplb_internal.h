@@ -20,6 +20,9 @@
 #define FEPLB_ST_COUNTS 2u     // counts passed to dispatch disagree with the ids
 #define FEPLB_ST_WAIT 4u       // a bounded mbarrier wait gave up inside the GEMM
 #define FEPLB_ST_GROUP 8u      // a group entry was malformed (expert or rows out of range)
+#define FEPLB_ST_PLAN 16u      // the GEMM's bounded wait for the planner's dynamic group table gave up
+#define FEPLB_WM_AUTO_ROWS_PER_EXPERT 768   // the weights-on-M form is the default below this many rows per expert
+#define FEPLB_WM_MAX_ENTRIES 1024    // group entries (static + dynamic table) one weights-on-M launch can hold
 
 int feplb_validate_config(const feplb_config* c);
 
@@ -45,7 +48,7 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
-                                     unsigned long long* counts_host_tagged, int32_t seq,
+                                     unsigned long long* counts_host_tagged, int32_t seq, unsigned long long* t_counts,
                                      cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
                               const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,
@@ -75,6 +78,24 @@ struct feplb_gemm_args {
 // One thread waits (bounded by limit_ns) on an mbarrier nobody completes; *gave_up = 1 and FEPLB_ST_WAIT expected.
 cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up, cudaStream_t st);
 int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
+// Weights-on-M form (feplb_gemm_wm.cu).  One launch per pass walks a.groups (filtered by a.which) and
+// then, if dyn.seq != 0, the planner's dynamic table, which it picks up on the device once the host-side
+// ready word carries (seq << 32) | number of groups; the CTA that wins `claim` copies it to table_dev.
+struct feplb_wm_dyn {
+  // the table travels as 32-byte entries {expert, row_start, rows, exec_rank, is_dynamic, seq, 0, 0}
+  void* table_dev = nullptr;                         // device copy of the table, written by the claiming CTA
+  const void* table_host = nullptr;                  // device address of the planner's table in mapped host memory
+  unsigned long long* ready_dev = nullptr;           // set by the claiming CTA after table_dev
+  const unsigned long long* ready_host = nullptr;    // device address of the word the planner thread sets after table_host
+  uint32_t* claim = nullptr;                         // device word the CTAs race for
+  uint32_t seq = 0;                                  // 0: no dynamic table
+  int max_groups = 0;                                // capacity of the tables
+  unsigned long long* stamps = nullptr;              // optional, 8 words: globaltimer marks of the two launches
+  unsigned long long wait_limit_ns = 0;              // bound of the wait for the table (0: the library's default)
+};
+bool feplb_wm_supported(int E, int d, int f, int n_entries_max);
+int feplb_launch_expert_ffn_wm(const feplb_gemm_args& a, const feplb_wm_dyn& dyn, cudaStream_t st, int64_t* n_launch,
+                               char* err, size_t errn);
 // ---- backward pass ---------------------------------------------------------------------------
 struct feplb_bwd_args {
   const void* x_perm; const void* ab_saved; void* h; void* d_y_perm;   // padding rows of h, d_y_perm, d_ab get zeros

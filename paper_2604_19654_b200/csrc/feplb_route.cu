@@ -160,7 +160,7 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
              int32_t* __restrict__ rank_load_out, int32_t* __restrict__ pad_off,
              feplb_group* __restrict__ groups, uint8_t* __restrict__ mask_out,
              int32_t* __restrict__ row_to_token, int64_t s_cap,
-             unsigned long long* __restrict__ counts_host_tagged, int32_t seq) {
+             unsigned long long* __restrict__ counts_host_tagged, int32_t seq, unsigned long long* t_counts) {
   __shared__ int tmp[64];
   __shared__ int sc[FEPLB_MAX_EXPERTS];
   const int e = threadIdx.x;
@@ -190,6 +190,11 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
     if (counts_host_tagged)
       *reinterpret_cast<volatile unsigned long long*>(counts_host_tagged + e) =
           ((unsigned long long)(uint32_t)seq << 32) | (uint32_t)c;
+  }
+  if (t_counts && e == 0) {            // timeline: when the counts left for the host (globaltimer, ns)
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    *t_counts = t;
   }
   int total;
   const int off = block_exclusive_scan((c + A - 1) / A * A, tmp, &total);   // also orders sc[] for all threads
@@ -489,7 +494,7 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
                                      int32_t* row_to_token, int64_t s_cap, uint32_t* status,
-                                     unsigned long long* counts_host_tagged, int32_t seq,
+                                     unsigned long long* counts_host_tagged, int32_t seq, unsigned long long* t_counts,
                                      cudaStream_t st, int64_t* n_launch) {
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
@@ -501,7 +506,7 @@ cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R
   }
   ++*n_launch;
   return launch(k_scan_fused, 1, 1024, 0, st, true, block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off,
-                groups, mask_out, row_to_token, s_cap, counts_host_tagged, seq);
+                groups, mask_out, row_to_token, s_cap, counts_host_tagged, seq, t_counts);
 }
 
 cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,

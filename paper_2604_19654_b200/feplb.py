@@ -19,7 +19,7 @@ OK, E_INVALID, E_RANGE, E_CUDA, E_NOMEM, E_TIMEOUT, E_STATE, E_DEVICE = 0, -1, -
 POLICY_LITERAL, POLICY_FIRST_FIT = 0, 1
 MASK_GIVEN, MASK_REACTIVE = 0, 1
 FFN_ALL, FFN_STATIC, FFN_DYNAMIC = 0, 1, 2
-FORM_AUTO, FORM_SINGLE, FORM_PAIR = -1, 0, 1
+FORM_AUTO, FORM_SINGLE, FORM_PAIR, FORM_WEIGHT_M = -1, 0, 1, 2
 HOST_SLOTS = 4            # staging sets of the pipelined host-buffer forward (FEPLB_HOST_SLOTS)
 
 
@@ -49,7 +49,8 @@ class Timeline(C.Structure):
         "host_upload_enqueued_us", "host_join_us", "host_return_us", "plan_us",
         "dev_hist_us", "dev_dispatch_us", "dev_static_ffn_us", "dev_dynamic_ffn_us", "dev_combine_us",
         "dev_counts_to_static_start_us", "dev_counts_to_static_end_us", "dev_total_us",
-        "dev_counts_to_copies_done_us", "phase2_copy_bytes")]
+        "dev_counts_to_copies_done_us", "phase2_copy_bytes",
+        "dev_ffn_pass1_us", "dev_ffn_pass2_us", "dev_plan_wait_us", "ffn_launches")]
 
 
 class FeplbError(RuntimeError):
@@ -108,6 +109,7 @@ def lib() -> C.CDLL:
             "feplb_moe_backward": (C.c_int, [vp] * 19 + [i32, vp]),
             "feplb_set_planner_timeout": (C.c_int, [vp, i32]),
             "feplb_set_gemm_form": (C.c_int, [vp, i32, i32]),
+            "feplb_set_planner_timing": (C.c_int, [vp, i32, i32]),
             "feplb_pack_weights": (C.c_int, [vp] * 8),
             "feplb_selftest_bounded_wait": (C.c_int, [vp, i32, vp]),
             "feplb_launch_count": (i64, [vp]),
@@ -408,6 +410,11 @@ class Context:
     def set_gemm_form(self, forward_form: int = FORM_AUTO, backward_pair: int = -1):
         """Forces the grouped-GEMM form (FORM_*) of the forward launches and the pair mask of the backward GEMMs."""
         self._chk(lib().feplb_set_gemm_form(self._h, int(forward_form), int(backward_pair)), "feplb_set_gemm_form")
+
+    def set_planner_timing(self, planner_delay_us: int = 0, device_wait_limit_us: int = 0):
+        """Test aid: delay the planner's table, bound the GEMM's device-side wait for it."""
+        self._chk(lib().feplb_set_planner_timing(self._h, int(planner_delay_us), int(device_wait_limit_us)),
+                  "feplb_set_planner_timing")
 
     def pack_weights(self, w1_in, w3_in, w2_in, w1, w3, w2, stream=None):
         """Input-major weights ([E,d,f], [E,d,f], [E,f,d]) -> the library's output-major layout."""

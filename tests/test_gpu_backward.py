@@ -41,6 +41,22 @@ def test_transpose_weights_bit_exact():
     case.close()
 
 
+def test_pack_weights_from_input_major_layout():
+    """feplb_pack_weights: [E,d,f] / [E,f,d] (x W as the operator is usually written) -> the library's layout."""
+    import torch
+    w = W.get_workload("cfg1").with_(E=3, d=384, f=192)
+    case = DeviceCase(w)
+    w1_in = F.bf16_tensor(np.ascontiguousarray(case.w1.transpose(0, 2, 1)))     # [E, d, f]
+    w3_in = F.bf16_tensor(np.ascontiguousarray(case.w3.transpose(0, 2, 1)))
+    w2_in = F.bf16_tensor(np.ascontiguousarray(case.w2.transpose(0, 2, 1)))     # [E, f, d]
+    w1, w3, w2 = torch.zeros_like(case.d_w1), torch.zeros_like(case.d_w3), torch.zeros_like(case.d_w2)
+    case.ctx.pack_weights(w1_in, w3_in, w2_in, w1, w3, w2)
+    torch.cuda.synchronize()
+    assert np.array_equal(F.bf16_bits(w1), case.w1) and np.array_equal(F.bf16_bits(w3), case.w3)
+    assert np.array_equal(F.bf16_bits(w2), case.w2)
+    case.close()
+
+
 def _run_backward(w, mb=0, scale=1.0, pair=-1, **cfg_kw):
     import torch
     case = DeviceCase(w, mb=mb, row_align=128, **cfg_kw)

@@ -162,7 +162,7 @@ def test_home_groups_match_the_no_move_plan():
 
 # ----------------------------------------------------------------------------- expert FFN
 
-def _ffn_case(E, d, f, rows_per_expert, A=1, seed=0, order=None):
+def _ffn_case(E, d, f, rows_per_expert, A=1, seed=0, order=None, form=None):
     """Builds x_perm / groups for the given per-expert row counts and checks H-free Y parity."""
     torch = _torch()
     rng = np.random.default_rng(seed)
@@ -171,6 +171,8 @@ def _ffn_case(E, d, f, rows_per_expert, A=1, seed=0, order=None):
     w = _tiny(max(int(counts.sum()), 1), 1, E, 1, d=d, f=f)
     cfg = F.config_from_workload(w, row_align=A)
     ctx = F.Context(cfg)
+    if form is not None:
+        ctx.set_gemm_form(form)
     cap = F.s_pad(cfg)
     xb = W.f32_to_bf16_bits((rng.standard_normal((cap, d)) * 0.5).astype(np.float32))
     w1 = W.f32_to_bf16_bits((rng.standard_normal((E, f, d)) / np.sqrt(d)).astype(np.float32))
@@ -210,6 +212,22 @@ def _ffn_case(E, d, f, rows_per_expert, A=1, seed=0, order=None):
 ])
 def test_expert_ffn_parity(E, d, f, rows):
     _ffn_case(E, d, f, rows)
+
+
+@pytest.mark.parametrize("form", [F.FORM_SINGLE, F.FORM_PAIR, F.FORM_WEIGHT_M])
+@pytest.mark.parametrize("E,d,f,rows", [
+    (1, 256, 128, [1]),                        # one row: a 16-row block, one chunk for half of the epilogue warps
+    (4, 256, 128, [0, 129, 0, 383]),           # empty experts; blocks of 144, 192 + 191 rows
+    (3, 512, 256, [16, 17, 33]),               # block sizes around the 16-row granule and the 32-row chunk
+    (2, 256, 384, [128, 256]),                 # exactly one small and one big unit per weight-tile pair
+    (5, 256, 128, [257, 31, 255, 513, 97]),    # alternating small / big units: both TMEM slot schemes in turn
+    (2, 2048, 768, [700, 45]),                 # the mid layer's shapes: 32 K blocks wrap the 3-stage ring many times
+    (2, 512, 128, [5000, 3]),                  # many blocks of one group, more units than CTAs in pass 2
+])
+def test_expert_ffn_parity_in_every_form(E, d, f, rows, form):
+    """Shapes every form supports (f % 128 == 0, d % 256 == 0), each form forced in turn."""
+    _ffn_case(E, d, f, rows, form=form)
+    _ffn_case(E, d, f, rows, A=128, form=form, order=list(range(E))[::-1])
 
 
 def test_expert_ffn_intermediates_within_rounding_of_the_oracle():
@@ -391,6 +409,94 @@ def test_forward_at_the_maximum_expert_count(A):
     w = W.get_workload("cfg2").with_(name="maxE", T=1500, E=1024, R=16, K=8, d=128, f=64, dyn=8, max_num_dyn=4, tau=1, alpha=0.3)
     case = DeviceCase(w, row_align=A)
     _check_forward(case, sample=200)
+    case.close()
+
+
+def _random_workload_wm(seed):
+    """Seeded random small layers in shapes the weights-on-M form takes (f % 128 == 0, d % 256 == 0)."""
+    rng = np.random.default_rng(5200 + seed)
+    R = int(rng.choice([1, 2, 3, 4]))
+    L = int(rng.choice([1, 2, 3, 5, 8]))
+    E = R * L
+    K = int(rng.integers(1, min(E, 8) + 1))
+    w = W.get_workload("cfg2").with_(
+        name=f"randwm{seed}", T=int(rng.integers(1, 1500)), E=E, R=R, K=K,
+        d=int(rng.choice([256, 512])), f=int(rng.choice([128, 256, 384])),
+        dyn=int(rng.integers(0, L + 1)), max_num_dyn=int(rng.integers(0, 4)), tau=int(rng.choice([0, 1, 8, 64])),
+        routing=str(rng.choice(["dirichlet", "zipf"])), alpha=float(rng.choice([0.2, 0.5, 1.2])))
+    return w, int(rng.choice([1, 128])), int(rng.integers(0, 2)), int(rng.integers(0, 2))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_forward_random_shapes_weights_on_m(seed):
+    """The whole layer with the weights-on-M form forced: one launch per pass runs the static groups
+    and then picks the planner's dynamic table up on the device.  Odd seeds also copy the migrated
+    experts' weights into receive slots (Phase 2)."""
+    w, A, split, phase2 = _random_workload_wm(seed)
+    case = DeviceCase(w, mb=seed, row_align=A, split=split, split_granule=128 if A == 128 else 16, phase2_copy=phase2)
+    case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case.ctx.set_timeline(bool(seed & 1))
+    _check_forward(case)
+    if seed & 1:
+        tl = case.ctx.get_timeline()
+        if phase2:                             # with weight copies the dynamic groups keep launches of their own
+            assert tl["ffn_launches"] == 4
+        else:
+            assert tl["ffn_launches"] == 2 and tl["dev_ffn_pass1_us"] > 0 and tl["dev_ffn_pass2_us"] > 0
+            assert tl["dev_counts_to_static_start_us"] > 0
+    # the same layer in the four-launch single-CTA form gives the same integers and an output within tolerance
+    out_wm = W.bf16_bits_to_f64(F.bf16_bits(case.buf.out))[: w.T].copy()
+    case.ctx.set_gemm_form(F.FORM_SINGLE)
+    _check_forward(case)
+    out_s = W.bf16_bits_to_f64(F.bf16_bits(case.buf.out))[: w.T]
+    assert np.abs(out_wm - out_s).max() <= 2e-2 * max(np.abs(out_s).max(), 1e-30)
+    case.close()
+
+
+def test_weights_on_m_form_is_refused_for_shapes_it_does_not_take():
+    case = DeviceCase(W.get_workload("cfg1"))                 # d = 128, f = 64
+    with pytest.raises(F.FeplbError) as ei:
+        case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    assert ei.value.code == F.E_INVALID
+    _check_forward(case)
+    case.close()
+
+
+def test_dynamic_table_arriving_late_is_waited_for_on_the_device(phase2=0):
+    """The planner is held back for 3 ms, far longer than the static groups take, so every CTA of the
+    merged launch runs out of static work and really waits for the table (bounded); results are
+    unchanged and the timeline shows the wait."""
+    w = W.get_workload("cfg2").with_(T=1024)
+    case = DeviceCase(w, mb=1, phase2_copy=phase2)
+    case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case.ctx.set_timeline(True)
+    case.ctx.set_planner_timing(planner_delay_us=3000)
+    p, _ = _check_forward(case)
+    assert len(p.moves) >= 1
+    tl = case.ctx.get_timeline()
+    assert tl["dev_plan_wait_us"] > 500, tl
+    case.ctx.set_planner_timing(0, 0)
+    _check_forward(case)
+    assert case.ctx.get_timeline()["dev_plan_wait_us"] < tl["dev_plan_wait_us"]
+    case.close()
+
+
+def test_device_wait_for_the_plan_expires_cleanly():
+    """The planner is held back for 150 ms while the GEMM's wait for its table is limited to 2 ms: the
+    kernels give up, skip the dynamic groups, raise the status bit and return; the forward call itself
+    succeeds (the plan did arrive on the host), feplb_check_status reports FEPLB_E_TIMEOUT, nothing
+    hangs and the next forward is correct."""
+    w = W.get_workload("cfg2").with_(T=1024)
+    case = DeviceCase(w, mb=1)
+    case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case.ctx.set_planner_timing(planner_delay_us=150000, device_wait_limit_us=2000)
+    case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
+    with pytest.raises(F.FeplbError) as ei:
+        case.ctx.check_status()
+    assert ei.value.code == F.E_TIMEOUT
+    case.ctx.set_planner_timing(0, 0)
+    case.ctx.check_status()
+    _check_forward(case)
     case.close()
 
 
