@@ -227,6 +227,7 @@ def run_cuda(args, w):
     cfg = F.config_from_workload(w, phase2_copy=1 if args.phase2 else 0, split=1 if args.split else 0)
     ctx = F.Context(cfg)
     ctx.set_gemm_form({"auto": F.FORM_AUTO, "single": F.FORM_SINGLE, "pair": F.FORM_PAIR, "weight_m": F.FORM_WEIGHT_M}[args.form])
+    ctx.set_launch_merging(args.merge)
     buf = F.Buffers(cfg)
 
     weights = W.gen_weights(w)
@@ -626,7 +627,7 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
         io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
         cold = getattr(args, "cold", None) or {}
         traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
-        roof = {"bound": "tensor", "kernel": "k_ffn_wm (weights on M, static + dynamic groups per launch)" if per_fw == 2 else "k_grouped_gemm",
+        roof = {"bound": "tensor", "kernel": ("k_grouped_gemm, static + dynamic groups per launch" if per_fw == 2 else "k_grouped_gemm") if args.form != "weight_m" else "k_ffn_wm",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak if achieved else None,
                 "peak_source": f"{peaks['source']} ({regime}: chosen from the SM clock and power-cap state sampled during this pass)",
@@ -753,6 +754,8 @@ def main():
     ap.add_argument("--max-repeats", type=int, default=400)
     ap.add_argument("--form", default="auto", choices=["auto", "single", "pair", "weight_m"],
                     help="grouped-GEMM form of the forward launches (feplb_set_gemm_form); auto is the library's choice")
+    ap.add_argument("--merge", type=int, default=-1, choices=[-1, 0, 1],
+                    help="feplb_set_launch_merging: 1 = one GEMM launch per pass over static then dynamic groups, 0 = four launches, -1 = library's choice")
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,

@@ -114,7 +114,7 @@ typedef struct {
   double dev_total_us;
   double dev_counts_to_copies_done_us;  /* device: counts copied -> Phase-2 weight copies landed (0 if none) */
   double phase2_copy_bytes;             /* bytes moved by those copies */
-  /* Weights-on-M form only (one launch per pass walks the static, then the dynamic groups); the
+  /* Merged launches only (one launch per pass walks the static, then the dynamic groups); the
    * marks are taken inside the kernels from the GPU's global timer.  There dev_static_ffn_us is the
    * whole expert FFN, dev_dynamic_ffn_us is 0, dev_counts_to_static_start_us ends at the first CTA's
    * start and dev_counts_to_static_end_us at the first moment a CTA ran out of static work. */
@@ -391,15 +391,24 @@ int feplb_set_planner_timeout(feplb_ctx* ctx, int32_t timeout_ms);
 /* Which form of the grouped-GEMM kernel the context uses.  forward_form: FEPLB_FORM_AUTO (default:
  * chosen from the geometry and, per group table, from the rows per group), FEPLB_FORM_SINGLE (one
  * CTA per 128-row tile), FEPLB_FORM_PAIR (clusters of two CTAs on 256-row tiles) or
- * FEPLB_FORM_WEIGHT_M (weight tiles on the M side, up to 256 rows of a group on the N side; in
- * feplb_moe_forward one launch per pass then runs the static groups and, after picking the
- * planner's table up on the device, the dynamic groups; needs f % 128 == 0, d % 256 == 0 and
- * 2*E + R*max_num_dyn <= 1024, else FEPLB_E_INVALID) for every forward launch.
+ * FEPLB_FORM_WEIGHT_M (weight tiles on the M side, up to 256 rows of a group on the N side; needs
+ * f % 128 == 0, d % 256 == 0 and 2*E + R*max_num_dyn <= 1024, else FEPLB_E_INVALID) for every
+ * forward launch.
  * backward_pair: -1 (default: chosen from the geometry) or a mask, bit 0 = activation-gradient
  * GEMMs in the pair form, bit 1 = weight-gradient GEMMs in the pair form.  Results do not depend
  * on the form beyond fp32 summation order.  Not allowed while a plan is pending. */
 int feplb_set_gemm_form(feplb_ctx* ctx, int32_t forward_form, int32_t backward_pair);
-/* Test and tuning aid for the weights-on-M form of feplb_moe_forward.  planner_delay_us: the
+/* How feplb_moe_forward launches the expert GEMMs.  merged = 1: one launch per pass runs the static
+ * groups (Section 2.3: while the CPU balancer works) and then the dynamic groups, whose table it
+ * picks up on the device with a bounded wait on a word the planner thread writes into mapped host
+ * memory -- two launches per forward, everything enqueued before the planner is joined, the
+ * static-first order kept inside each launch.  merged = 0: static and dynamic groups in launches of
+ * their own (four per forward), the dynamic ones enqueued after the planner has been joined and
+ * each table in the form that suits it.  -1 (default): merged while a forward's groups are small
+ * (below ~768 rows per expert).  With cfg.phase2_copy the four-launch order is always used.
+ * merged = 1 needs 2*E + R*max_num_dyn <= 1024.  Not allowed while a plan is pending. */
+int feplb_set_launch_merging(feplb_ctx* ctx, int32_t merged);
+/* Test and tuning aid for the merged launches of feplb_moe_forward.  planner_delay_us: the
  * planner thread sleeps that long before it publishes its table (0 = off), so that the GEMM's
  * device-side wait for the table really is entered.  device_wait_limit_us: bound of that wait
  * (0 = the default, 400 ms); when it expires the kernels skip the dynamic groups, raise a status

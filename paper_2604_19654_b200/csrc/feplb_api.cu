@@ -25,7 +25,7 @@ inline double us_since(clk::time_point t0) {
   return std::chrono::duration<double, std::micro>(clk::now() - t0).count();
 }
 enum JobState { JOB_IDLE = 0, JOB_PENDING = 1, JOB_RUNNING = 2, JOB_DONE = 3 };
-enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_COPIES, EV_N };
+enum { EV_T0 = 0, EV_HIST, EV_DISPATCH, EV_STATIC0, EV_STATIC1, EV_DYN0, EV_DYN1, EV_COMBINE, EV_COUNTS, EV_COPIES, EV_STAMPS, EV_N };
 constexpr int kEvRing = 16;   // forwards whose stage events may be outstanding
 constexpr int kStampWords = 16;   // [0..3] pass 1, [4..7] pass 2 (see WmParams::stamps), [8] counts left the device
 }  // namespace
@@ -44,6 +44,10 @@ struct feplb_ctx {
   bool wm_ok = false;          // the weights-on-M form supports this geometry
   bool wm = false;             // ... and is the form in use (feplb_create's choice or feplb_set_gemm_form)
   bool wm_auto = false;
+  bool merged_ok = false;      // both group tables of a forward fit one launch (static, then dynamic groups)
+  bool merged = false;         // ... and feplb_moe_forward runs that way: two GEMM launches instead of four
+  bool merged_auto = false;
+  bool merged_pair = false;    // form of the merged launches when none is forced
   int32_t planner_delay_us = 0;        // test aid: the planner sleeps before it publishes its table
   int32_t device_wait_limit_us = 0;    // bound of the GEMM's wait for the table (0: default)
   // weights-on-M form: the words through which a running GEMM launch learns that the dynamic table exists
@@ -316,6 +320,8 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   c->s_cap = feplb_s_pad(cfg);
   // 256-row pair tiles pay off when an expert's segment is several tiles long on average
   c->gemm_pair_auto = c->gemm_pair_default = (int64_t)cfg->T * cfg->K >= (int64_t)2048 * cfg->E;
+  // a merged launch runs static and dynamic groups in one form: the two-CTA form from 256 rows per expert
+  c->merged_pair = (int64_t)cfg->T * cfg->K >= (int64_t)256 * cfg->E;
   // backward GEMMs: the pair form pays once an expert's segment spans several 256-row tiles
   // (measured: -7.5 % backward time at 1024 rows per expert, slower at 384)
   c->bwd_pair_auto = c->bwd_pair = (int64_t)cfg->T * cfg->K >= (int64_t)512 * cfg->E ? 3 : 0;
@@ -327,7 +333,14 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
   // the L2 port once per 256 rows); from ~1000 rows per expert the two-CTA form keeps its lead because
   // it can overlap every tile's epilogue with the next tile's MMAs.
   c->wm_ok = feplb_wm_supported(cfg->E, cfg->d, cfg->f, cfg->E + cap_groups);
-  c->wm_auto = c->wm = c->wm_ok && S < (int64_t)FEPLB_WM_AUTO_ROWS_PER_EXPERT * cfg->E;
+  c->wm_auto = c->wm = false;      // measured a few percent behind the tokens-on-M forms at every benchmarked size: on request only
+  // One launch per pass over the static and then the dynamic groups (the table of the latter is
+  // picked up on the device): saves two launch ramps and two partly filled last waves per forward,
+  // which matters while a forward's GEMMs take a few hundred microseconds; one form serves both
+  // tables then, so it stays off where the dynamic groups want the two-CTA form and the static ones
+  // do not (from ~1000 rows per expert).
+  c->merged_ok = cfg->E + cap_groups <= FEPLB_MAX_GROUPS;
+  c->merged_auto = c->merged = c->merged_ok && S < (int64_t)FEPLB_WM_AUTO_ROWS_PER_EXPERT * cfg->E;
   bool ok = true;
   ok = ok && cudaMalloc(&c->d_dyn_ready, 2 * sizeof(unsigned long long)) == cudaSuccess &&     // [0] ready word, [1] claim word
        cudaMemset(c->d_dyn_ready, 0, 2 * sizeof(unsigned long long)) == cudaSuccess;
@@ -530,8 +543,7 @@ static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void
     const feplb_wm_dyn none;
     return feplb_launch_expert_ffn_wm(a, dyn ? *dyn : none, st, &c->launches, c->err, sizeof(c->err));
   }
-  if (dyn) return fail(c, FEPLB_E_STATE, "expert_ffn: merged launch without the weights-on-M form");
-  return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err));
+  return feplb_launch_expert_ffn(a, st, &c->launches, c->err, sizeof(c->err), dyn);
 }
 
 extern "C" int feplb_expert_ffn(feplb_ctx* c, const void* x_perm, const void* w1, const void* w3, const void* w2,
@@ -634,6 +646,7 @@ static int harvest_slot(feplb_ctx* c, int r) {
   if (!c->ev_used[r]) return FEPLB_OK;
   cudaEvent_t* ev = c->evr[r];
   CUDA_TRY(c, cudaEventSynchronize(ev[EV_COMBINE]));
+  if (c->ev_host[r].ffn_launches == 2) CUDA_TRY(c, cudaEventSynchronize(ev[EV_STAMPS]));
   float ms = 0;
   auto el = [&](cudaEvent_t a, cudaEvent_t b) { return cudaEventElapsedTime(&ms, a, b) == cudaSuccess ? ms * 1e3 : 0.0; };
   feplb_timeline t = c->ev_host[r];
@@ -706,17 +719,13 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   // Not with Phase-2 weight copies: the dynamic groups would then wait, inside a kernel that holds
   // every SM, for device-to-device copies that the driver may carry out with kernels of its own;
   // that case keeps the four-launch order (the dynamic launches follow the copies in stream order).
-  const bool wm = c->wm && !g.phase2_copy;
+  const bool wm = c->merged && !g.phase2_copy;
   c->tl.ffn_launches = wm ? 2 : 4;
   c->tl.dev_ffn_pass1_us = c->tl.dev_ffn_pass2_us = c->tl.dev_plan_wait_us = 0;
   unsigned long long* stamps = nullptr;
   if (wm && c->timeline_on) {
     stamps = c->d_stamps + (size_t)c->ev_slot * kStampWords;
     CUDA_TRY(c, cudaMemsetAsync(stamps, 0xFF, sizeof(unsigned long long) * kStampWords, st));
-#ifdef FEPLB_PROBE
-    CUDA_TRY(c, cudaMemsetAsync(stamps + 10, 0, 8, st));
-    CUDA_TRY(c, cudaMemsetAsync(stamps + 12, 0, 8, st));
-#endif
   }
   TL_EVENT(EV_T0);
   // step 1: counts, rank loads, segment offsets and the home group table in two launches; the
@@ -765,20 +774,20 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     dyn.seq = (uint32_t)seq; dyn.max_groups = c->plan.cap_groups; dyn.stamps = stamps;
     dyn.wait_limit_ns = 1000ull * (unsigned long long)c->device_wait_limit_us;
     if (rc == FEPLB_OK)
-      rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st, -1, &dyn);
+      rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st,
+                    c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (int)c->merged_pair, &dyn);
     TL_EVENT(EV_STATIC1);
     c->tl.host_enqueue_static_done_us = us_since(c->t0);
     TL_EVENT(EV_DYN0);
     TL_EVENT(EV_DYN1);
     int rc_comb = rc == FEPLB_OK ? feplb_combine(c, y_perm, slot_to_row, gates, out, stream) : FEPLB_OK;
-    if (stamps && rc == FEPLB_OK && rc_comb == FEPLB_OK) {
-      cudaError_t e = cudaMemcpyAsync(c->h_stamps + (size_t)c->ev_slot * kStampWords, stamps,
-                                      sizeof(unsigned long long) * kStampWords, cudaMemcpyDeviceToHost, st);
-      if (e != cudaSuccess) rc_comb = fail(c, FEPLB_E_CUDA, "timeline copy: %s", cudaGetErrorString(e));
-    }
     if (c->timeline_on && rc == FEPLB_OK && rc_comb == FEPLB_OK) {
       cudaError_t e = cudaEventRecord(c->ev[EV_COMBINE], st);
-      if (e != cudaSuccess) rc_comb = fail(c, FEPLB_E_CUDA, "event record: %s", cudaGetErrorString(e));
+      if (e == cudaSuccess && stamps)      // the kernels' own marks follow the last stage event to the host
+        e = cudaMemcpyAsync(c->h_stamps + (size_t)c->ev_slot * kStampWords, stamps, sizeof(unsigned long long) * kStampWords,
+                            cudaMemcpyDeviceToHost, st);
+      if (e == cudaSuccess) e = cudaEventRecord(c->ev[EV_STAMPS], st);
+      if (e != cudaSuccess) rc_comb = fail(c, FEPLB_E_CUDA, "timeline records: %s", cudaGetErrorString(e));
     }
     // join the planner (always, so that the context returns to idle): everything is already enqueued
     int rc_join = join_planner(c, c->planner_timeout_ms + 500, plan_copy);
@@ -958,12 +967,15 @@ extern "C" int feplb_set_gemm_form(feplb_ctx* c, int32_t forward_form, int32_t b
   return FEPLB_OK;
 }
 
-#ifdef FEPLB_PROBE
-extern "C" int feplb_probe_stamps(feplb_ctx* c, unsigned long long* out) {
-  for (int i = 0; i < kStampWords; ++i) out[i] = c->h_stamps[(size_t)c->ev_slot * kStampWords + i];
-  return 0;
+extern "C" int feplb_set_launch_merging(feplb_ctx* c, int32_t merged) {
+  if (!c || merged < -1 || merged > 1) return FEPLB_E_INVALID;
+  if (merged == 1 && !c->merged_ok)
+    return fail(c, FEPLB_E_INVALID, "set_launch_merging: needs 2*E + R*max_num_dyn <= %d", FEPLB_MAX_GROUPS);
+  std::lock_guard<std::mutex> lk(c->mu);
+  if (c->job != JOB_IDLE) return fail(c, FEPLB_E_STATE, "set_launch_merging: a plan is pending");
+  c->merged = merged < 0 ? c->merged_auto : merged != 0;
+  return FEPLB_OK;
 }
-#endif
 
 extern "C" int feplb_set_planner_timing(feplb_ctx* c, int32_t planner_delay_us, int32_t device_wait_limit_us) {
   if (!c || planner_delay_us < 0 || planner_delay_us > 1000000 || device_wait_limit_us < 0) return FEPLB_E_INVALID;

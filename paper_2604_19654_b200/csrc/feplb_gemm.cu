@@ -22,6 +22,7 @@
 
 #include "feplb_internal.h"
 #include "feplb_tc.cuh"
+#include "feplb_dyn.cuh"
 
 namespace {
 
@@ -62,8 +63,11 @@ struct SmemTail {
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kAccStages];
   unsigned long long tmem_empty[kAccStages];
+  unsigned long long dyn_bar;         // completed by warp 0 once the dynamic entries are in place
   uint32_t tmem_base;
   int abort_flag;
+  int n_entries;                      // entries in use (the table known at launch, then the planner's dynamic groups)
+  int total_mtiles;                   // prefix[n_entries]
   int prefix[FEPLB_MAX_GROUPS + 1];   // prefix[g] = M tiles of groups before g
   int g_row_start[FEPLB_MAX_GROUPS];
   int g_rows[FEPLB_MAX_GROUPS];
@@ -89,6 +93,9 @@ struct GemmParams {
   int ld_out;           // elements between output rows
   uint32_t* status;
   __nv_bfloat16* ab_out;   // pass 1, optional: pre-activations a | b saved for the backward pass ([rows, 2f])
+  DynTable dyn;            // the planner's table of dynamic groups, walked after `groups` (dyn.seq == 0: none in this launch)
+  unsigned long long* stamps;   // optional, preset to all ones, globaltimer ns: [0] first CTA's start, [1] first time a CTA
+                                // ran out of static tiles, [2] ~(last CTA's end), [3] ~(longest wait for the dynamic table)
 };
 
 
@@ -182,6 +189,45 @@ __device__ __forceinline__ void stage_and_store(uint32_t stg, const uint32_t* pa
   __syncwarp();
 }
 
+// One entry of a group table -> shared-memory arrays; returns its number of M tiles (0 if not selected).
+template <int kRows>
+__device__ __forceinline__ int put_group(SmemTail* t, int idx, int expert, int row_start, int rows, int is_dynamic, bool selected,
+                                         const GemmParams& p) {
+  int tiles = 0;
+  if (selected && rows > 0) {
+    const bool ok = expert >= 0 && expert < p.E && row_start >= 0 && (int64_t)row_start + rows <= p.s_cap &&
+                    is_dynamic - 2 < p.n_recv_slots;
+    if (ok) tiles = (rows + kRows - 1) / kRows;
+    else atomicOr(p.status, FEPLB_ST_GROUP);
+  }
+  t->g_row_start[idx] = row_start;
+  t->g_rows[idx] = rows;
+  // expert id in the low half; receive slot + 1 in the high half (0 = weights at home)
+  t->g_expert[idx] = (expert & 0xffff) | ((is_dynamic >= 2 ? is_dynamic - 1 : 0) << 16);
+  return tiles;
+}
+
+// In-place inclusive scan of t->prefix[first+1 .. first+n] (tile counts) by one warp; prefix[first] is the base.
+__device__ __forceinline__ void warp_scan_prefix(SmemTail* t, int first, int n, int lane) {
+  const int per = (n + 31) / 32;
+  const int g0 = min(n, lane * per), g1 = min(n, g0 + per);
+  int sum = 0;
+  for (int g = g0; g < g1; ++g) sum += t->prefix[first + g + 1];
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  int run = t->prefix[first] + incl - sum;
+  __syncwarp();
+  for (int g = g0; g < g1; ++g) {
+    run += t->prefix[first + g + 1];
+    t->prefix[first + g + 1] = run;
+  }
+  __syncwarp();
+}
+
 template <bool SWIGLU, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
@@ -222,6 +268,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       // one arrival per epilogue warp (of both CTAs in the pair form: the leader's barrier collects them)
       mbar_init(smem_u32(&tail->tmem_empty[a]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
+    mbar_init(smem_u32(&tail->dyn_bar), 1);
     tail->abort_flag = 0;
     fence_barrier_init();
   }
@@ -238,60 +285,89 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // everything above touched only this CTA's resources; from here on the results of the kernels
   // before this one (rows, group table) are read
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (p.stamps && threadIdx.x == 0) atomicMin(&p.stamps[0], global_timer_ns());
   for (int g = threadIdx.x; g < p.n_groups; g += kThreads) {
     const feplb_group gr = p.groups[g];
     const bool selected = p.which == FEPLB_FFN_ALL || (p.which == FEPLB_FFN_STATIC) == (gr.is_dynamic == 0);
-    int tiles = 0;
-    if (selected && gr.rows > 0) {
-      const bool ok = gr.expert >= 0 && gr.expert < p.E && gr.row_start >= 0 &&
-                      (int64_t)gr.row_start + gr.rows <= p.s_cap && gr.is_dynamic - 2 < p.n_recv_slots;
-      if (ok) tiles = (gr.rows + kTileRows - 1) / kTileRows;
-      else atomicOr(p.status, FEPLB_ST_GROUP);
-    }
-    tail->prefix[g + 1] = tiles;   // turned into a prefix sum below
-    tail->g_row_start[g] = gr.row_start;
-    tail->g_rows[g] = gr.rows;
-    // expert id in the low half; receive slot + 1 in the high half (0 = weights at home)
-    tail->g_expert[g] = (gr.expert & 0xffff) | ((gr.is_dynamic >= 2 ? gr.is_dynamic - 1 : 0) << 16);
+    tail->prefix[g + 1] = put_group<kTileRows>(tail, g, gr.expert, gr.row_start, gr.rows, gr.is_dynamic, selected, p);   // scanned below
   }
+  if (threadIdx.x == 0) tail->prefix[0] = 0;
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
-    // exclusive scan of the per-group tile counts, 32 lanes x contiguous chunks
-    const int per = (p.n_groups + 31) / 32;
-    const int g0 = lane * per, g1 = min(p.n_groups, g0 + per);
-    int sum = 0;
-    for (int g = g0; g < g1; ++g) sum += tail->prefix[g + 1];
-    int incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += y;
+    warp_scan_prefix(tail, 0, p.n_groups, lane);
+    if (lane == 0) {
+      tail->n_entries = p.n_groups;
+      tail->total_mtiles = tail->prefix[p.n_groups];
     }
-    int run = incl - sum;
-    for (int g = g0; g < g1; ++g) {
-      const int t = tail->prefix[g + 1];
-      run += t;
-      tail->prefix[g + 1] = run;
-    }
-    if (lane == 0) tail->prefix[0] = 0;
   }
   __syncthreads();
   if (PAIR) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = tail->tmem_base;
-  const int total_tiles = tail->prefix[p.n_groups] * p.n_tiles_n;
+  const bool has_dyn = p.dyn.seq != 0;
+  const int n_static_entries = p.n_groups;
+  const int n_static_tiles = tail->prefix[p.n_groups] * p.n_tiles_n;
   const uint32_t b_half_bytes = (uint32_t)p.bn * BK * 2;
   const uint32_t stage_tx = PAIR ? 2 * (kABytes + b_half_bytes) : kABytes + 2 * b_half_bytes;
 
   if (warp == 0) {
-    // ---- TMA producer ---------------------------------------------------------------------
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
-        const TileCoord c = tile_coord<kTileRows>(tail, p.n_groups, p.n_tiles_n, tile);
+    // ---- TMA producer (lane 0 issues; the whole warp fetches the dynamic table) ----------------
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true, dyn_known = !has_dyn;
+    int n_entries = n_static_entries, total = n_static_tiles;
+    // Reads the n_dyn groups of the dynamic table from its device copy, appends its entries and tells
+    // the other roles; false if an entry does not carry this forward's sequence number yet.
+    auto take_table = [&](int n_dyn) -> bool {
+      if (n_dyn < 0 || n_static_entries + n_dyn > FEPLB_MAX_GROUPS) {
+        if (lane == 0) atomicOr(p.status, FEPLB_ST_GROUP);
+        n_dyn = 0;
+      }
+      bool good = true;
+      for (int i = lane; i < n_dyn; i += 32) {
+        int e, rs, rw, dy;
+        if (!dyn_entry(p.dyn, i, e, rs, rw, dy)) { good = false; continue; }
+        tail->prefix[n_static_entries + i + 1] = put_group<kTileRows>(tail, n_static_entries + i, e, rs, rw, dy, true, p);
+      }
+      if (!__all_sync(0xffffffffu, good)) return false;
+      warp_scan_prefix(tail, n_static_entries, n_dyn, lane);
+      n_entries = n_static_entries + n_dyn;
+      total = tail->prefix[n_entries] * p.n_tiles_n;
+      if (lane == 0) {
+        tail->n_entries = n_entries;
+        tail->total_mtiles = tail->prefix[n_entries];
+        mbar_arrive(smem_u32(&tail->dyn_bar));      // release: the entries above are visible to the waiters
+      }
+      dyn_known = true;
+      return true;
+    };
+    bool claimer = false, tried_claim = false;
+    for (int tile = worker; ok; tile += n_workers) {
+      if (!dyn_known && tile >= total) {
+        // Out of static tiles: now the table is needed (bounded wait; see feplb_dyn.cuh).
+        const unsigned long long t0 = global_timer_ns();
+        if (p.stamps && lane == 0) atomicMin(&p.stamps[1], t0);
+        while (!dyn_known) {
+          const int n_dyn = dyn_wait_table(p.dyn, lane, abort_flag, p.status, t0, claimer, tried_claim);
+          if (n_dyn == kDynAbort) { ok = false; break; }
+          // no table within the limit: go on as if it were empty, so that the static tiles still in
+          // flight in this CTA complete normally; the status word carries the reason
+          if (!take_table(n_dyn == kDynGaveUp ? 0 : n_dyn) && global_timer_ns() - t0 > p.dyn.wait_limit_ns + kWaitLimitNs) {
+            if (lane == 0) atomicOr(p.status, FEPLB_ST_PLAN);
+            take_table(0);
+          }
+        }
+        if (!ok) break;
+        if (p.stamps && lane == 0) atomicMin(&p.stamps[3], ~(global_timer_ns() - t0));
+      }
+      if (tile >= total) break;
+      const TileCoord c = tile_coord<kTileRows>(tail, n_entries, p.n_tiles_n, tile);
+      // While static tiles remain, peek at the device-side word once per tile: the load is in flight
+      // during the K loop below and is looked at after it, so it costs the pipeline nothing.
+      unsigned long long peek = 0;
+      if (!dyn_known && lane == 0) peek = ld_relaxed_gpu_u64(p.dyn.ready_dev);
+      if (lane == 0) {
         // weights of a migrated expert come from its slot of the receive buffer
         const CUtensorMap* mb0 = c.slot >= 0 ? &tm_r0 : &tm_b0;
         const CUtensorMap* mb1 = c.slot >= 0 ? &tm_r1 : &tm_b1;
@@ -323,10 +399,15 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
-        // leave time for copies already issued to land before the CTA's shared memory goes away
-        for (int i = 0; i < 2000; ++i) __nanosleep(100);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (ok && !dyn_known) {
+        peek = __shfl_sync(0xffffffffu, peek, 0);
+        if (dyn_peek_count(p.dyn, peek) >= 0) take_table(dyn_peek_count(p.dyn, peek));
       }
+    }
+    if (!ok && lane == 0) {
+      // leave time for copies already issued to land before the CTA's shared memory goes away
+      for (int i = 0; i < 2000; ++i) __nanosleep(100);
     }
   } else if (warp == 1) {
     // ---- MMA issuer -------------------------------------------------------------------------
@@ -334,8 +415,16 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       const uint32_t idesc = make_idesc(kTileRows, 2 * p.bn);
       int stage = 0, as = 0;
       uint32_t phase = 0, aphase = 0;
-      bool ok = true;
-      for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
+      bool ok = true, dyn_known = !has_dyn;
+      int total = n_static_tiles;
+      for (int tile = worker; ok; tile += n_workers) {
+        if (tile >= total) {
+          if (dyn_known) break;
+          if (!(ok = mbar_wait(smem_u32(&tail->dyn_bar), 0, abort_flag, p.status, p.dyn.wait_limit_ns + 2 * kWaitLimitNs))) break;
+          dyn_known = true;
+          total = tail->total_mtiles * p.n_tiles_n;
+          if (tile >= total) break;
+        }
         if (!(ok = mbar_wait(smem_u32(&tail->tmem_empty[as]), aphase ^ 1u, abort_flag, p.status))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * kAccCols);
@@ -374,9 +463,20 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int out_cols = SWIGLU ? p.bn : 2 * p.bn;
     int as = 0;
     uint32_t aphase = 0;
-    bool ok = true;
-    for (int tile = worker; ok && tile < total_tiles; tile += n_workers) {
-      const TileCoord c = tile_coord<kTileRows>(tail, p.n_groups, p.n_tiles_n, tile);
+    bool ok = true, dyn_known = !has_dyn;
+    int n_entries = n_static_entries, total = n_static_tiles;
+    for (int tile = worker; ok; tile += n_workers) {
+      if (tile >= total) {
+        if (dyn_known) break;
+        ok = mbar_wait(smem_u32(&tail->dyn_bar), 0, abort_flag, p.status, p.dyn.wait_limit_ns + 2 * kWaitLimitNs);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        dyn_known = true;
+        n_entries = tail->n_entries;
+        total = tail->total_mtiles * p.n_tiles_n;
+        if (tile >= total) break;
+      }
+      const TileCoord c = tile_coord<kTileRows>(tail, n_entries, p.n_tiles_n, tile);
       ok = mbar_wait(smem_u32(&tail->tmem_full[as]), aphase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -439,6 +539,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // ---- teardown ---------------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (p.stamps && threadIdx.x == 0) atomicMin(&p.stamps[2], ~global_timer_ns());
   if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory: leave together
   if (warp == 1) {
     __syncwarp();
@@ -539,8 +640,13 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUte
 
 }  // namespace
 
-int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn) {
-  if (a.n_groups == 0 || a.s_cap == 0) return FEPLB_OK;
+int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn,
+                            const feplb_wm_dyn* dyn) {
+  if ((a.n_groups == 0 && !(dyn && dyn->seq)) || a.s_cap == 0) return FEPLB_OK;
+  if (dyn && a.n_groups + dyn->max_groups > FEPLB_MAX_GROUPS) {
+    snprintf(err, errn, "expert_ffn: the two group tables of a merged launch exceed %d entries", FEPLB_MAX_GROUPS);
+    return FEPLB_E_INVALID;
+  }
   // pass 1: H = silu(X W1) * (X W3);  N tile = bn columns of H, MMA N = 2*bn
   const int bn1 = (a.f % 128 == 0) ? 128 : 64;
   // pass 2: Y = H W2;  N tile = 2*bn columns of Y
@@ -570,9 +676,13 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
   p1.n_tiles_n = a.f / bn1; p1.num_k_blocks = a.d / BK; p1.b_rows_per_expert = a.f; p1.bn = bn1;
   p1.out = (__nv_bfloat16*)a.h; p1.ld_out = a.f; p1.status = a.status; p1.ab_out = (__nv_bfloat16*)a.ab_out;
+  const feplb_wm_dyn none;
+  p1.dyn = feplb_dyn_table(dyn ? *dyn : none);
+  p1.stamps = dyn ? dyn->stamps : nullptr;
   GemmParams p2 = p1;
   p2.n_tiles_n = a.d / (2 * bn2); p2.num_k_blocks = a.f / BK; p2.b_rows_per_expert = a.d; p2.bn = bn2;
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d; p2.ab_out = nullptr;
+  p2.stamps = p1.stamps ? p1.stamps + 4 : nullptr;
 
   cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st)
                          : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st);

@@ -77,10 +77,9 @@ struct feplb_gemm_args {
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).
 // One thread waits (bounded by limit_ns) on an mbarrier nobody completes; *gave_up = 1 and FEPLB_ST_WAIT expected.
 cudaError_t feplb_launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, int* gave_up, cudaStream_t st);
-int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn);
-// Weights-on-M form (feplb_gemm_wm.cu).  One launch per pass walks a.groups (filtered by a.which) and
-// then, if dyn.seq != 0, the planner's dynamic table, which it picks up on the device once the host-side
-// ready word carries (seq << 32) | number of groups; the CTA that wins `claim` copies it to table_dev.
+// A launch per pass walks a.groups (filtered by a.which) and then, if dyn.seq != 0, the planner's dynamic
+// table, which it picks up on the device once the host-side ready word carries (seq << 32) | number of
+// groups; the CTA that wins `claim` copies it to table_dev (feplb_dyn.cuh).
 struct feplb_wm_dyn {
   // the table travels as 32-byte entries {expert, row_start, rows, exec_rank, is_dynamic, seq, 0, 0}
   void* table_dev = nullptr;                         // device copy of the table, written by the claiming CTA
@@ -93,6 +92,10 @@ struct feplb_wm_dyn {
   unsigned long long* stamps = nullptr;              // optional, 8 words: globaltimer marks of the two launches
   unsigned long long wait_limit_ns = 0;              // bound of the wait for the table (0: the library's default)
 };
+// Tokens-on-M forms (feplb_gemm.cu): single CTA per 128-row tile or, with a.pair, clusters of two on 256-row tiles.
+int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* n_launch, char* err, size_t errn,
+                            const feplb_wm_dyn* dyn = nullptr);
+// Weights-on-M form (feplb_gemm_wm.cu).
 bool feplb_wm_supported(int E, int d, int f, int n_entries_max);
 int feplb_launch_expert_ffn_wm(const feplb_gemm_args& a, const feplb_wm_dyn& dyn, cudaStream_t st, int64_t* n_launch,
                                char* err, size_t errn);

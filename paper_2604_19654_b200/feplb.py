@@ -110,6 +110,7 @@ def lib() -> C.CDLL:
             "feplb_set_planner_timeout": (C.c_int, [vp, i32]),
             "feplb_set_gemm_form": (C.c_int, [vp, i32, i32]),
             "feplb_set_planner_timing": (C.c_int, [vp, i32, i32]),
+            "feplb_set_launch_merging": (C.c_int, [vp, i32]),
             "feplb_pack_weights": (C.c_int, [vp] * 8),
             "feplb_selftest_bounded_wait": (C.c_int, [vp, i32, vp]),
             "feplb_launch_count": (i64, [vp]),
@@ -410,6 +411,10 @@ class Context:
     def set_gemm_form(self, forward_form: int = FORM_AUTO, backward_pair: int = -1):
         """Forces the grouped-GEMM form (FORM_*) of the forward launches and the pair mask of the backward GEMMs."""
         self._chk(lib().feplb_set_gemm_form(self._h, int(forward_form), int(backward_pair)), "feplb_set_gemm_form")
+
+    def set_launch_merging(self, merged: int = -1):
+        """1: one GEMM launch per pass over static, then dynamic groups; 0: launches of their own; -1: library's choice."""
+        self._chk(lib().feplb_set_launch_merging(self._h, int(merged)), "feplb_set_launch_merging")
 
     def set_planner_timing(self, planner_delay_us: int = 0, device_wait_limit_us: int = 0):
         """Test aid: delay the planner's table, bound the GEMM's device-side wait for it."""

@@ -44,7 +44,7 @@ def test_transpose_weights_bit_exact():
 def test_pack_weights_from_input_major_layout():
     """feplb_pack_weights: [E,d,f] / [E,f,d] (x W as the operator is usually written) -> the library's layout."""
     import torch
-    w = W.get_workload("cfg1").with_(E=3, d=384, f=192)
+    w = W.get_workload("cfg1").with_(E=4, d=384, f=192)
     case = DeviceCase(w)
     w1_in = F.bf16_tensor(np.ascontiguousarray(case.w1.transpose(0, 2, 1)))     # [E, d, f]
     w3_in = F.bf16_tensor(np.ascontiguousarray(case.w3.transpose(0, 2, 1)))

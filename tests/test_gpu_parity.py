@@ -390,7 +390,10 @@ def test_forward_random_shapes(seed):
     w, A, split, pair = _random_workload(seed)
     case = DeviceCase(w, mb=seed, row_align=A, split=split, split_granule=128 if A == 128 else 16)
     case.ctx.set_gemm_form(F.FORM_PAIR if pair else F.FORM_SINGLE)
+    case.ctx.set_launch_merging((seed >> 1) & 1)      # both launch orders: four launches, or two that pick the plan up on the device
+    case.ctx.set_timeline(True)
     _check_forward(case)
+    assert case.ctx.get_timeline()["ffn_launches"] == (2 if (seed >> 1) & 1 else 4)
     case.close()
 
 
@@ -435,6 +438,7 @@ def test_forward_random_shapes_weights_on_m(seed):
     w, A, split, phase2 = _random_workload_wm(seed)
     case = DeviceCase(w, mb=seed, row_align=A, split=split, split_granule=128 if A == 128 else 16, phase2_copy=phase2)
     case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case.ctx.set_launch_merging(1)
     case.ctx.set_timeline(bool(seed & 1))
     _check_forward(case)
     if seed & 1:
@@ -462,13 +466,15 @@ def test_weights_on_m_form_is_refused_for_shapes_it_does_not_take():
     case.close()
 
 
-def test_dynamic_table_arriving_late_is_waited_for_on_the_device(phase2=0):
+@pytest.mark.parametrize("form", [F.FORM_SINGLE, F.FORM_PAIR, F.FORM_WEIGHT_M])
+def test_dynamic_table_arriving_late_is_waited_for_on_the_device(form):
     """The planner is held back for 3 ms, far longer than the static groups take, so every CTA of the
     merged launch runs out of static work and really waits for the table (bounded); results are
     unchanged and the timeline shows the wait."""
     w = W.get_workload("cfg2").with_(T=1024)
-    case = DeviceCase(w, mb=1, phase2_copy=phase2)
-    case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case = DeviceCase(w, mb=1)
+    case.ctx.set_gemm_form(form)
+    case.ctx.set_launch_merging(1)
     case.ctx.set_timeline(True)
     case.ctx.set_planner_timing(planner_delay_us=3000)
     p, _ = _check_forward(case)
@@ -481,14 +487,16 @@ def test_dynamic_table_arriving_late_is_waited_for_on_the_device(phase2=0):
     case.close()
 
 
-def test_device_wait_for_the_plan_expires_cleanly():
+@pytest.mark.parametrize("form", [F.FORM_SINGLE, F.FORM_PAIR, F.FORM_WEIGHT_M])
+def test_device_wait_for_the_plan_expires_cleanly(form):
     """The planner is held back for 150 ms while the GEMM's wait for its table is limited to 2 ms: the
     kernels give up, skip the dynamic groups, raise the status bit and return; the forward call itself
     succeeds (the plan did arrive on the host), feplb_check_status reports FEPLB_E_TIMEOUT, nothing
     hangs and the next forward is correct."""
     w = W.get_workload("cfg2").with_(T=1024)
     case = DeviceCase(w, mb=1)
-    case.ctx.set_gemm_form(F.FORM_WEIGHT_M)
+    case.ctx.set_gemm_form(form)
+    case.ctx.set_launch_merging(1)
     case.ctx.set_planner_timing(planner_delay_us=150000, device_wait_limit_us=2000)
     case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf)
     with pytest.raises(F.FeplbError) as ei:
