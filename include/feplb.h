@@ -178,6 +178,29 @@ int feplb_plan(const feplb_config* cfg, const int32_t* counts, const uint8_t* dy
 int feplb_ema_update(double* ema, const int32_t* counts, int32_t E, double decay);
 int feplb_place_experts(const double* load, int32_t E, int32_t R, int32_t* new_index);
 
+/* Expert parallelism over R real ranks (Section 2.2, Phases 1 and 2; Section 2.3: every device
+ * derives the same plan by itself from the counts all devices know after Phase 1).  Host logic
+ * only: the row exchange and the peer copies themselves are the caller's (no multi-GPU data plane
+ * is part of this library yet).  Rank s holds its own tokens; counts_by_src[s*E + e] is the number
+ * of its (token, k) slots routed to expert e -- the R x E matrix every rank has after one
+ * all-gather of its row.  From it every rank computes, identically:
+ *   - counts[e] = sum_s counts_by_src[s][e] and the plan of feplb_plan on them (written to *plan);
+ *     the rows of expert e are ordered by source rank, then by slot, which is the order
+ *     feplb_dispatch gives when the ranks' tokens are numbered one rank after the other;
+ *   - Phase 1, dispatch all-to-all-v: rank s sends counts_by_src[s][e] rows to home(e);
+ *   - Phase 2: for move i (expert, src = home, dst, rows) the first not yet moved `rows` rows of
+ *     the expert's segment and the expert's three weight matrices go from src to slot
+ *     dst*max_num_dyn + (number of earlier moves into dst) of dst's receive buffer;
+ *   - Combine: every executed row returns from the rank that ran it straight to its source rank.
+ * Outputs for `rank` (host arrays of R entries each, any may be NULL): rows it sends to / receives
+ * from every rank in Phase 1, in Phase 2 and in the combine; copies[0..*n_copies) lists ALL weight
+ * copies in move order (cap_copies >= R*max_num_dyn always suffices; FEPLB_E_NOMEM otherwise). */
+typedef struct { int32_t expert, src, dst, slot, rows; int64_t weight_bytes; } feplb_weight_copy;
+int feplb_ep_schedule(const feplb_config* cfg, const int32_t* counts_by_src, const uint8_t* dyn_mask, int32_t rank,
+                      feplb_plan_out* plan, int64_t* p1_send, int64_t* p1_recv, int64_t* p2_send, int64_t* p2_recv,
+                      int64_t* comb_send, int64_t* comb_recv, feplb_weight_copy* copies, int32_t cap_copies,
+                      int32_t* n_copies);
+
 /* ---- device steps ------------------------------------------------------------------------- */
 
 /* Step 0, optional (Section 2.3, router; Section 3.1, top-k routing without auxiliary loss):

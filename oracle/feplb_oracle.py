@@ -50,6 +50,11 @@ place_experts   macro-level expert-to-device assignment from historical load (Se
                 Predictor; no algorithm given): capacity-constrained LPT greedy, a reading.
                 PARITY UNPINNED against the paper; pinned: permutation invariant, brute-force
                 optimum and the 4/3 LPT bound on tiny inputs
+ep_exchange     who sends how many rows to whom when the R ranks are real devices (Section 2.2, Phase 1:
+                tokens go to their expert's home; Phase 2: the rows of migrated pieces go on to the
+                receiving device with the expert's weights; Section 2.3: results return to the source
+                devices), counted one row at a time from a plan.  A bookkeeping definition.  pinned:
+                conservation laws, a hand-worked case
 moe_layer_backward  gradients of the layer w.r.t. x, gates and the expert weights (Table 2 reports
                 backward times; the pass itself is not described): the chain rule of the forward
                 definition.                                               pinned: central finite
@@ -353,6 +358,49 @@ def combine(y_rows: np.ndarray, slot_to_row: np.ndarray, gates: np.ndarray) -> n
     for k in range(K):
         out += g[:, k:k + 1] * y_rows[slot_to_row[:, k]]
     return out
+
+
+# ----------------------------------------------------------------------------- expert parallelism over real ranks
+
+def ep_exchange(counts_by_src, plan_result, max_num_dyn: int):
+    """Row traffic of expert parallelism over R real ranks for one micro-batch (Sections 2.2, 2.3).
+
+    ``counts_by_src[s][e]`` = slots of rank s's own tokens routed to expert e.  The rows of expert e
+    are ordered by source rank, then by slot (the order ``permute`` gives when the ranks' tokens are
+    numbered one rank after the other); ``plan_result`` is ``plan()`` on the column sums.  Every row
+    is followed on its way: source -> home of its expert (Phase 1) -> the rank that executes it, if
+    its piece was migrated (Phase 2) -> back to the source (combine).  Returns
+    (p1, p2, comb, copies): p1[s][r], p2[s][r], comb[s][r] = rows rank s sends to rank r in the three
+    steps, copies = [(expert, src, dst, slot, rows)] with slot = dst*max_num_dyn + (earlier moves
+    into dst).
+    """
+    cbs = [[int(v) for v in row] for row in np.asarray(counts_by_src).tolist()]
+    R, E = len(cbs), len(cbs[0])
+    L = E // R
+    p1 = [[0] * R for _ in range(R)]
+    p2 = [[0] * R for _ in range(R)]
+    comb = [[0] * R for _ in range(R)]
+    for e in range(E):
+        exec_of_row = []
+        for (ge, _start, rows, exec_rank, _dyn) in plan_result["groups"]:
+            if ge == e:
+                exec_of_row += [exec_rank] * rows
+        assert len(exec_of_row) == sum(cbs[s][e] for s in range(R))
+        pos = 0
+        for s in range(R):
+            for _ in range(cbs[s][e]):
+                home, x = e // L, exec_of_row[pos]
+                pos += 1
+                p1[s][home] += 1
+                if x != home:
+                    p2[home][x] += 1
+                comb[x][s] += 1
+    used = [0] * R
+    copies = []
+    for (e, src, dst, rows) in plan_result["moves"]:
+        copies.append((e, src, dst, dst * max_num_dyn + used[dst], rows))
+        used[dst] += 1
+    return np.array(p1, np.int64), np.array(p2, np.int64), np.array(comb, np.int64), copies
 
 
 # ----------------------------------------------------------------------------- whole layer

@@ -2,6 +2,7 @@
 // per-micro-batch load balancer (paper Section 2.3).  Pure C++, no CUDA: the planner thread of
 // the library and callers without a GPU run exactly this code.
 #include <algorithm>
+#include <climits>
 #include <cstdint>
 #include <vector>
 
@@ -137,6 +138,66 @@ extern "C" int feplb_plan(const feplb_config* cfg, const int32_t* counts, const 
     off += ((int64_t)counts[e] + A - 1) / A * A;
   }
   out->n_groups = n_groups;
+  return FEPLB_OK;
+}
+
+extern "C" int feplb_ep_schedule(const feplb_config* cfg, const int32_t* counts_by_src, const uint8_t* dyn_mask, int32_t rank,
+                                 feplb_plan_out* plan, int64_t* p1_send, int64_t* p1_recv, int64_t* p2_send, int64_t* p2_recv,
+                                 int64_t* comb_send, int64_t* comb_recv, feplb_weight_copy* copies, int32_t cap_copies,
+                                 int32_t* n_copies) {
+  int rc = feplb_validate_config(cfg);
+  if (rc != FEPLB_OK) return rc;
+  if (!counts_by_src || !dyn_mask || !plan || rank < 0 || rank >= cfg->R) return FEPLB_E_INVALID;
+  const int E = cfg->E, R = cfg->R, L = E / R;
+  std::vector<int32_t> counts(E, 0);
+  for (int s = 0; s < R; ++s)
+    for (int e = 0; e < E; ++e) {
+      const int32_t c = counts_by_src[(size_t)s * E + e];
+      if (c < 0 || (int64_t)counts[e] + c > INT32_MAX) return FEPLB_E_INVALID;
+      counts[e] += c;
+    }
+  if ((rc = feplb_plan(cfg, counts.data(), dyn_mask, plan)) != FEPLB_OK) return rc;
+  auto zero = [&](int64_t* a) { if (a) std::fill(a, a + R, (int64_t)0); };
+  zero(p1_send); zero(p1_recv); zero(p2_send); zero(p2_recv); zero(comb_send); zero(comb_recv);
+  // Phase 1: every source sends each expert's rows to the expert's home
+  for (int e = 0; e < E; ++e) {
+    if (p1_send) p1_send[e / L] += counts_by_src[(size_t)rank * E + e];
+    if (p1_recv && e / L == rank)
+      for (int s = 0; s < R; ++s) p1_recv[s] += counts_by_src[(size_t)s * E + e];
+  }
+  // Phase 2 and the combine: walk every expert's segment piece by piece (moved pieces from the
+  // front, in move order, then the home remainder) and split each piece by source rank
+  std::vector<int> next_slot(R, 0);
+  int nc = 0;
+  for (int i = 0; i < plan->n_moves; ++i) {
+    const feplb_move& m = plan->moves[i];
+    if (p2_send && m.src == rank) p2_send[m.dst] += m.rows;
+    if (p2_recv && m.dst == rank) p2_recv[m.src] += m.rows;
+    if (copies) {
+      if (nc >= cap_copies) return FEPLB_E_NOMEM;
+      copies[nc] = feplb_weight_copy{m.expert, m.src, m.dst, m.dst * cfg->max_num_dyn + next_slot[m.dst],
+                                     m.rows, (int64_t)3 * cfg->d * cfg->f * 2};
+    }
+    ++next_slot[m.dst];
+    ++nc;
+  }
+  if (n_copies) *n_copies = nc;
+  std::vector<int64_t> seg_pos(E, 0);              // rows of expert e already handed out
+  for (int gi = 0; gi < plan->n_groups; ++gi) {
+    const feplb_group& g = plan->groups[gi];       // groups of one expert come in segment order
+    const int e = g.expert;
+    int64_t a = seg_pos[e], b = a + g.rows, off = 0;
+    seg_pos[e] = b;
+    for (int s = 0; s < R; ++s) {                  // source s owns [off, off + c) of the segment
+      const int64_t c = counts_by_src[(size_t)s * E + e];
+      const int64_t lo = std::max(a, off), hi = std::min(b, off + c);
+      if (hi > lo) {
+        if (comb_send && g.exec_rank == rank) comb_send[s] += hi - lo;
+        if (comb_recv && s == rank) comb_recv[g.exec_rank] += hi - lo;
+      }
+      off += c;
+    }
+  }
   return FEPLB_OK;
 }
 

@@ -53,6 +53,10 @@ class Timeline(C.Structure):
         "dev_ffn_pass1_us", "dev_ffn_pass2_us", "dev_plan_wait_us", "ffn_launches")]
 
 
+class WeightCopy(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("expert", "src", "dst", "slot", "rows")] + [("weight_bytes", C.c_int64)]
+
+
 class FeplbError(RuntimeError):
     def __init__(self, code: int, where: str, detail: str = ""):
         self.code = code
@@ -82,6 +86,8 @@ def lib() -> C.CDLL:
             "feplb_s_pad": (C.c_size_t, [C.POINTER(Config)]),
             "feplb_select_dynamic": (C.c_int, [C.POINTER(i64), i32, i32, i32, C.POINTER(C.c_uint8)]),
             "feplb_plan": (C.c_int, [C.POINTER(Config), C.POINTER(i32), C.POINTER(C.c_uint8), C.POINTER(PlanOut)]),
+            "feplb_ep_schedule": (C.c_int, [C.POINTER(Config), C.POINTER(i32), C.POINTER(C.c_uint8), i32, C.POINTER(PlanOut)] +
+                                  [C.POINTER(i64)] * 6 + [C.POINTER(WeightCopy), i32, C.POINTER(i32)]),
             "feplb_ema_update": (C.c_int, [C.POINTER(C.c_double), C.POINTER(i32), i32, C.c_double]),
             "feplb_place_experts": (C.c_int, [C.POINTER(C.c_double), i32, i32, C.POINTER(i32)]),
             "feplb_route_topk": (C.c_int, [vp, vp, vp, vp, vp]),
@@ -212,6 +218,33 @@ def plan(cfg: Config, counts, dyn_mask) -> Plan:
     if rc:
         raise FeplbError(rc, "feplb_plan")
     return p
+
+
+def ep_schedule(cfg: Config, counts_by_src, dyn_mask, rank: int) -> dict:
+    """What ``rank`` of R real expert-parallel ranks sends and receives (host only; see feplb_ep_schedule).
+
+    ``counts_by_src`` int32 [R, E]: the all-gathered per-rank expert counts.  Returns the plan (identical on
+    every rank), int64 [R] row counts ``p1_send/p1_recv`` (dispatch), ``p2_send/p2_recv`` (migrated rows),
+    ``comb_send/comb_recv`` (combine) and ``copies``: every weight copy (expert, src, dst, slot, rows, bytes).
+    """
+    cbs = np.ascontiguousarray(counts_by_src, np.int32)
+    msk = np.ascontiguousarray(dyn_mask, np.uint8)
+    if cbs.shape != (cfg.R, cfg.E) or msk.shape != (cfg.E,):
+        raise ValueError("counts_by_src must be [R, E] and dyn_mask [E]")
+    p = Plan(cfg)
+    arr = {k: np.zeros(cfg.R, np.int64) for k in ("p1_send", "p1_recv", "p2_send", "p2_recv", "comb_send", "comb_recv")}
+    cap = max(1, cfg.R * cfg.max_num_dyn)
+    copies = (WeightCopy * cap)()
+    n = C.c_int32()
+    rc = lib().feplb_ep_schedule(C.byref(cfg), cbs.ctypes.data_as(C.POINTER(C.c_int32)), msk.ctypes.data_as(C.POINTER(C.c_uint8)),
+                                 int(rank), C.byref(p.c), *[a.ctypes.data_as(C.POINTER(C.c_int64)) for a in arr.values()],
+                                 copies, cap, C.byref(n))
+    if rc:
+        raise FeplbError(rc, "feplb_ep_schedule")
+    out = dict(arr)
+    out["plan"] = p
+    out["copies"] = [(c.expert, c.src, c.dst, c.slot, c.rows, c.weight_bytes) for c in copies[: n.value]]
+    return out
 
 
 def dispatch_noalloc(cfg: Config, x, topk_ids, counts, x_perm, slot_to_row, row_to_token, status=None, stream=None):

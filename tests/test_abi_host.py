@@ -144,6 +144,30 @@ def test_select_dynamic_matches_oracle(R, L, dyn, seed):
     assert np.array_equal(F.select_dynamic(score, R * L, R, dyn), O.select_dynamic(score, R * L, R, dyn))
 
 
+@settings(max_examples=150, deadline=None)
+@given(st.sampled_from([1, 2, 3, 4, 8]), st.integers(1, 6), st.integers(0, 2 ** 31), st.integers(0, 4), st.sampled_from([0, 1]))
+def test_ep_schedule_matches_the_oracle_row_by_row_count(R, L, seed, mnd, split):
+    """feplb_ep_schedule (interval arithmetic on the plan's pieces) against the oracle's ep_exchange,
+    which follows every row: all six send/receive vectors of every rank, the plan and the weight copies."""
+    rng = np.random.default_rng(seed)
+    E = R * L
+    cbs = (rng.dirichlet(np.full(E, 0.4), size=R) * rng.integers(0, 600, size=(R, 1))).astype(np.int32)
+    mask = (rng.random(E) < 0.7).astype(np.uint8)
+    cfg = F.make_config(T=1, K=1, E=E, R=R, d=128, f=64, max_num_dyn=mnd, tau=int(rng.choice([0, 8])), split=split, split_granule=16)
+    counts = cbs.sum(0)
+    op = O.plan(counts, mask, R, tau=cfg.tau, max_num_dyn=mnd, split=split, split_granule=16)
+    p1, p2, comb, copies = O.ep_exchange(cbs, op, mnd)
+    for rank in range(R):
+        s = F.ep_schedule(cfg, cbs, mask, rank)
+        assert s["plan"].moves == [tuple(int(v) for v in m) for m in op["moves"]]
+        assert s["plan"].groups == [tuple(int(v) for v in g) for g in op["groups"]]
+        assert np.array_equal(s["p1_send"], p1[rank]) and np.array_equal(s["p1_recv"], p1[:, rank])
+        assert np.array_equal(s["p2_send"], p2[rank]) and np.array_equal(s["p2_recv"], p2[:, rank])
+        assert np.array_equal(s["comb_send"], comb[rank]) and np.array_equal(s["comb_recv"], comb[:, rank])
+        assert [c[:5] for c in s["copies"]] == copies
+        assert all(c[5] == 3 * 128 * 64 * 2 for c in s["copies"])
+
+
 def test_plan_capacity_error():
     cfg = F.make_config(T=1, K=1, E=4, R=2, d=128, f=64, max_num_dyn=2, tau=1)
     p = F.Plan(cfg)

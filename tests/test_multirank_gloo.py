@@ -95,3 +95,124 @@ def test_dyn_sensitivity_is_monotone_and_reactive_mask_beats_fixed():
     fixed, _ = bench.plan_sensitivity(w, 4, mask="fixed", n_mb=4)
     literal, _ = bench.plan_sensitivity(w, 4, policy=0, n_mb=4)
     assert fixed < r4 and literal <= r4 and a4 < 1.2
+
+
+# ----------------------------------------------------------------------------- expert parallelism over real ranks
+
+def _ep_worker(rank, world, port, q):
+    """One rank of a real expert-parallel group on CPU.  Control plane: the library's (all-gather of
+    the counts + feplb_ep_schedule).  Data plane: replayed on numpy arrays through object
+    collectives, with the oracle's FFN on the rows each rank executes."""
+    from oracle import feplb_oracle as O
+    from paper_2604_19654_b200 import ep, feplb as F, workloads as W
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    R = world
+    w = W.get_workload("cfg1").with_(name="ep", T=48 * R, E=4 * R, R=R, K=3, dyn=2, max_num_dyn=2, tau=1, alpha=1.4)
+    x, ids, gates = W.gen_microbatch(w, 7)                       # the whole micro-batch, seeded: every rank draws the same
+    w1, w3, w2 = W.gen_weights(w)
+    T_loc, L = w.T // R, w.E // R
+    t0 = rank * T_loc                                            # this rank's tokens: [t0, t0 + T_loc)
+    my_ids, my_x, my_g = ids[t0:t0 + T_loc], x[t0:t0 + T_loc], gates[t0:t0 + T_loc]
+    cfg = F.config_from_workload(w)
+    # ---- control plane
+    local_counts = np.bincount(my_ids.ravel(), minlength=w.E).astype(np.int32)
+    cbs = ep.exchange_counts(local_counts)
+    sch = ep.schedule(cfg, cbs, rank)
+    plan = sch["plan"]
+    # ---- Phase 1: every slot's row to the home of its expert, in (source rank, slot) order
+    out_p1 = [[] for _ in range(R)]
+    for s_loc in range(T_loc * w.K):
+        e = int(my_ids.ravel()[s_loc])
+        out_p1[e // L].append((e, rank, s_loc, my_x[s_loc // w.K]))
+    assert [len(v) for v in out_p1] == sch["p1_send"].tolist()
+    everything = [None] * R
+    dist.all_gather_object(everything, out_p1)
+    seg = {e: [] for e in range(rank * L, (rank + 1) * L)}      # expert -> rows in segment order
+    for src in range(R):
+        assert len(everything[src][rank]) == sch["p1_recv"][src]
+        for (e, s, s_loc, row) in everything[src][rank]:
+            seg[e].append((s, s_loc, row))
+    # ---- Phase 2: migrated pieces (rows + the expert's weights) from the home to the receiving rank
+    out_p2 = [[] for _ in range(R)]
+    taken = {e: 0 for e in seg}
+    for (e, src, dst, slot, rows, nbytes) in sch["copies"]:
+        if src == rank:
+            piece = seg[e][taken[e]:taken[e] + rows]
+            taken[e] += rows
+            out_p2[dst].append((e, slot, piece, (w1[e], w3[e], w2[e])))
+    assert [sum(len(m[2]) for m in v) for v in out_p2] == sch["p2_send"].tolist()
+    dist.all_gather_object(everything, out_p2)
+    work = [(e, rows[taken[e]:], (w1[e], w3[e], w2[e])) for e, rows in seg.items()]      # home remainders, home weights
+    slots_seen = []
+    for src in range(R):
+        got = everything[src][rank]
+        assert sum(len(m[2]) for m in got) == sch["p2_recv"][src]
+        for (e, slot, piece, wts) in got:
+            assert nbytes == 3 * w.d * w.f * 2 and slot // cfg.max_num_dyn == rank
+            slots_seen.append(slot)
+            work.append((e, piece, wts))                        # weights as they arrived in the receive slot
+    assert len(set(slots_seen)) == len(slots_seen)
+    assert sum(len(rows) for _, rows, _ in work) == int(plan.load_after[rank])
+    # ---- expert FFN on the rows this rank executes, then the combine: results straight back to the sources
+    out_c = [[] for _ in range(R)]
+    for (e, rows, (a1, a3, a2)) in work:
+        if not rows:
+            continue
+        xb = np.stack([r[2] for r in rows])
+        y = O.expert_ffn(xb, np.zeros(len(rows), np.int64), a1[None], a3[None], a2[None])
+        for (s, s_loc, _), yr in zip(rows, y):
+            out_c[s].append((s_loc, yr))
+    assert [len(v) for v in out_c] == sch["comb_send"].tolist()
+    dist.all_gather_object(everything, out_c)
+    y_slots = np.zeros((T_loc * w.K, w.d))
+    for src in range(R):
+        assert len(everything[src][rank]) == sch["comb_recv"][src]
+        for (s_loc, yr) in everything[src][rank]:
+            y_slots[s_loc] = yr
+    out = O.combine(y_slots, np.arange(T_loc * w.K).reshape(T_loc, w.K), my_g)
+    ref = O.moe_layer(x, ids, gates, w1, w3, w2, w.E, tokens=np.arange(t0, t0 + T_loc))
+    err = float(np.abs(out - ref).max() / np.abs(ref).max())
+    summary = (plan.moves, plan.groups, plan.load_before.tolist(), plan.load_after.tolist(), sch["copies"])
+    gathered = [None] * R
+    dist.all_gather_object(gathered, (summary, sch["p1_send"].tolist(), sch["p1_recv"].tolist(), sch["p2_send"].tolist(),
+                                      sch["p2_recv"].tolist(), sch["comb_send"].tolist(), sch["comb_recv"].tolist(), err))
+    dist.barrier()
+    q.put((rank, gathered))
+    dist.destroy_process_group()
+
+
+def _run_ep(world):
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_ep_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=300) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    return res[0][1]
+
+
+def _check_ep(world):
+    g = _run_ep(world)
+    summaries = [r[0] for r in g]
+    assert all(s == summaries[0] for s in summaries)            # every rank derived the same plan and copy list
+    moves, _, before, after, copies = summaries[0]
+    assert len(moves) >= 1 and max(after) < max(before)
+    for name, (snd, rcv) in {"phase 1": (1, 2), "phase 2": (3, 4), "combine": (5, 6)}.items():
+        send = np.array([r[snd] for r in g])                    # send[s][r]
+        recv = np.array([r[rcv] for r in g])                    # recv[r][s]
+        assert np.array_equal(send, recv.T), name               # what s sends to r is what r expects from s
+    assert np.array([r[3] for r in g]).sum() == sum(m[3] for m in moves)
+    assert max(r[7] for r in g) < 1e-12                         # the replayed layer equals the oracle's
+
+
+def test_expert_parallel_protocol_world_2():
+    _check_ep(2)
+
+
+def test_expert_parallel_protocol_world_4():
+    _check_ep(4)

@@ -578,3 +578,40 @@ def test_backward_against_finite_differences():
         for idx in [tuple(rng.integers(0, n) for n in arr.shape) for _ in range(6)]:
             assert grad[idx] == pytest.approx(fd(arr, idx, pos), rel=1e-5, abs=1e-7)
     assert O.dsilu(np.array([0.0]))[0] == 0.5 and O.dsilu(np.array([40.0]))[0] == pytest.approx(1.0)
+
+
+# ----------------------------------------------------------------------------- expert parallelism over real ranks
+
+def test_ep_exchange_conservation_and_handworked_case():
+    """ep_exchange against what must hold whatever the plan is, and against a case small enough to
+    follow by hand."""
+    # hand-worked: R = 2, L = 2.  Rank 0's tokens send 3 rows to e0, 1 to e2; rank 1's send 2 to e0, 1 to e1, 2 to e3.
+    cbs = np.array([[3, 0, 1, 0], [2, 1, 0, 2]])
+    counts = cbs.sum(0)                                        # [5, 1, 1, 2] -> loads [6, 3]
+    p = O.plan(counts, [1, 1, 1, 1], 2, tau=1, max_num_dyn=2)
+    assert p["moves"] == [(1, 0, 1, 1)]                        # gap 3: e0 (5) does not fit, e1 (1 row) moves 0 -> 1
+    p1, p2, comb, copies = O.ep_exchange(cbs, p, 2)
+    assert p1.tolist() == [[3, 1], [3, 2]]                     # to home: e0/e1 live on rank 0, e2/e3 on rank 1
+    assert p2.tolist() == [[0, 1], [0, 0]]                     # the one row of e1 goes on from rank 0 to rank 1
+    assert comb.tolist() == [[3, 2], [1, 3]]                   # rank 0 ran e0 (3 rows of rank 0, 2 of rank 1); rank 1 ran e2, e3 and e1's row
+    assert copies == [(1, 0, 1, 2, 1)]                         # slot = dst * max_num_dyn + 0
+    # conservation on random inputs
+    rng = np.random.default_rng(31)
+    for _ in range(30):
+        R = int(rng.choice([2, 3, 4]))
+        L = int(rng.choice([1, 2, 4]))
+        cbs = rng.integers(0, 40, size=(R, R * L))
+        counts = cbs.sum(0)
+        mask = (rng.random(R * L) < 0.7).astype(np.uint8)
+        mnd = int(rng.integers(0, 3))
+        p = O.plan(counts, mask, R, tau=int(rng.choice([0, 5])), max_num_dyn=mnd)
+        p1, p2, comb, copies = O.ep_exchange(cbs, p, mnd)
+        assert np.array_equal(p1.sum(1), cbs.sum(1))           # every slot leaves its source once
+        assert np.array_equal(p1.sum(0), counts.reshape(R, L).sum(1))      # and arrives at its expert's home
+        assert np.array_equal(comb.sum(0), cbs.sum(1))         # every slot comes back to its source
+        assert np.array_equal(comb.sum(1), p["load_after"])    # from the rank that executed it
+        assert p2.sum() == sum(m[3] for m in p["moves"]) and not np.diag(p2).any()
+        assert np.array_equal(p1.sum(0) - p2.sum(1) + p2.sum(0), p["load_after"])
+        assert [c[:3] + (c[4],) for c in copies] == [tuple(m) for m in p["moves"]]
+        slots = [c[3] for c in copies]
+        assert len(set(slots)) == len(slots) and all(c[2] * mnd <= c[3] < (c[2] + 1) * mnd for c in copies)
