@@ -71,10 +71,11 @@ typedef struct {
   int32_t split_granule;    /* rows; pieces of a cut expert are multiples of it */
   int32_t row_align;        /* A: expert segments of the permuted buffers start at multiples of A */
   int32_t mask_policy;      /* FEPLB_MASK_*: who chooses the dynamic experts in feplb_moe_forward */
-  int32_t phase2_copy;      /* 1: feplb_moe_forward really copies the weights of every migrated expert
-                               into a receive buffer of R*max_num_dyn slots (Section 2.2, Phase 2;
-                               Section 2.3, memory paragraph) with copy-engine transfers that overlap
-                               the static-expert GEMM, and the dynamic GEMM reads them from there.
+  int32_t phase2_copy;      /* 1: feplb_moe_forward really copies, for every migrated piece, the expert's
+                               weights into a receive buffer of R*max_num_dyn slots and the piece's rows
+                               into a receive region (Section 2.2, Phase 2: tokens and weights; Section
+                               2.3, memory paragraph) with device-to-device transfers that overlap the
+                               static-expert GEMM, and the dynamic GEMM reads both from there.
                                0 (default): a migration only relabels the executing rank. */
 } feplb_config;
 
@@ -84,7 +85,8 @@ typedef struct { int32_t expert, src, dst, rows; } feplb_move;
 /* One segment of the grouped GEMM: rows [row_start, row_start + rows) of the permuted buffers
  * belong to `expert` and are executed on virtual rank `exec_rank`.  is_dynamic: 0 = static expert,
  * 1 = dynamic expert computed with its home weights, 2 + s = dynamic expert whose weights are read
- * from slot s of the context's receive buffer (phase2_copy). */
+ * from slot s of the context's receive buffer and whose rows are read from the context's receive
+ * region of rows, at the same row numbers (phase2_copy). */
 typedef struct { int32_t expert, row_start, rows, exec_rank, is_dynamic; } feplb_group;
 
 /* Caller-sized plan.  cap_moves >= R*max_num_dyn and cap_groups >= E + R*max_num_dyn always

@@ -73,6 +73,10 @@ struct feplb_ctx {
   void* d_recv_w3 = nullptr;
   void* d_recv_w2 = nullptr;
   int n_recv_slots = 0;
+  void* d_recv_x = nullptr;    // Phase-2 receive region of the migrated pieces' rows: [s_cap, d], same row numbers as x_perm
+  cudaEvent_t ev_gather = nullptr;          // the permuted rows of the current forward are written
+  std::atomic<int32_t> gather_seq{0};       // ... recorded for the forward with this sequence number
+  const void* job_x_perm = nullptr;
   void* d_preact = nullptr;   // caller-owned [s_cap, 2f]: pass 1 saves a | b there when set (training)
   // pinned staging
   int32_t* h_counts = nullptr;
@@ -229,6 +233,29 @@ void planner_main(feplb_ctx* c) {
             next_move[gr.expert] = i + 1;
             if (i < c->plan.n_moves) gr.is_dynamic = 2 + move_slot[i];
           }
+          // ... and so do the rows of the moved pieces (Section 2.2: Phase 2 redistributes tokens and
+          // weights): each piece's rows go to the same row numbers of the receive region, once the
+          // gather kernel of this forward has written them (the event is recorded by the calling thread,
+          // which then publishes the forward's sequence number)
+          if (ce == cudaSuccess && c->plan.n_moves > 0 && c->job_x_perm) {
+            const auto g0 = clk::now();
+            while (c->gather_seq.load(std::memory_order_acquire) != c->job_flag_seq &&
+                   std::chrono::duration<double>(clk::now() - g0).count() < 1e-3 * c->planner_timeout_ms) {
+#if defined(__x86_64__) || defined(__i386__)
+              __builtin_ia32_pause();
+#endif
+            }
+            if (c->gather_seq.load(std::memory_order_acquire) != c->job_flag_seq) ce = cudaErrorNotReady;
+            if (ce == cudaSuccess) ce = cudaStreamWaitEvent(c->copy_stream, c->ev_gather, 0);
+            const size_t row_bytes = (size_t)cfg.d * 2;
+            for (int g = 0; g < n && ce == cudaSuccess; ++g) {
+              const feplb_group& gr = c->h_dyn_groups[g];
+              if (gr.is_dynamic < 2 || gr.rows <= 0) continue;
+              ce = cudaMemcpyAsync((char*)c->d_recv_x + row_bytes * gr.row_start, (const char*)c->job_x_perm + row_bytes * gr.row_start,
+                                   row_bytes * gr.rows, cudaMemcpyDeviceToDevice, c->copy_stream);
+              c->copy_bytes += (double)row_bytes * gr.rows;
+            }
+          }
           if (ce == cudaSuccess && c->copy_bytes > 0) ce = cudaEventRecord(c->ev[EV_COPIES], c->copy_stream);
           if (ce != cudaSuccess) c->copy_bytes = 0;
           c->tl.phase2_copy_bytes = c->copy_bytes;
@@ -367,6 +394,8 @@ extern "C" int feplb_create(const feplb_config* cfg, feplb_ctx** out) {
     ok = ok && cudaMalloc(&c->d_recv_w1, per * n) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_recv_w3, per * n) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_recv_w2, per * n) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_recv_x, (size_t)(c->s_cap > 0 ? c->s_cap : 1) * cfg->d * 2) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_gather, cudaEventDisableTiming) == cudaSuccess;
   }
   ok = ok && cudaMallocHost(&c->h_counts, sizeof(int32_t) * cfg->E) == cudaSuccess;
   ok = ok && cudaHostAlloc(&c->h_dyn_groups, (sizeof(feplb_group) * cap_groups + 15) / 16 * 16, cudaHostAllocMapped) == cudaSuccess &&
@@ -428,6 +457,8 @@ extern "C" int feplb_destroy(feplb_ctx* c) {
   cudaFree(c->d_recv_w1);
   cudaFree(c->d_recv_w3);
   cudaFree(c->d_recv_w2);
+  cudaFree(c->d_recv_x);
+  if (c->ev_gather) cudaEventDestroy(c->ev_gather);
   cudaFree(c->d_dyn_ready);
   cudaFree(c->d_dyn_tab32);
   cudaFreeHost(c->h_dyn_tab32);
@@ -539,6 +570,7 @@ static int ffn_impl(feplb_ctx* c, const void* x_perm, const void* w1, const void
   a.status = c->d_status; a.num_sms = c->num_sms; a.pair = pair;
   a.ab_out = c->d_preact;
   a.recv_w1 = c->d_recv_w1; a.recv_w3 = c->d_recv_w3; a.recv_w2 = c->d_recv_w2; a.n_recv_slots = c->n_recv_slots;
+  a.recv_x = c->d_recv_x;
   if (c->wm && n_groups + (dyn ? dyn->max_groups : 0) <= FEPLB_WM_MAX_ENTRIES) {
     const feplb_wm_dyn none;
     return feplb_launch_expert_ffn_wm(a, dyn ? *dyn : none, st, &c->launches, c->err, sizeof(c->err));
@@ -749,6 +781,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
                                        (int64_t)c->s_cap, c->d_status, c->h_counts_tagged, seq,
                                        stamps ? stamps + 8 : nullptr, st, &c->launches));
   c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
+  c->job_x_perm = x_perm;
   if ((rc = plan_kick_flag(c, dyn_mask_host, seq, wm)) != FEPLB_OK) return rc;
   TL_EVENT(EV_COUNTS);
   TL_EVENT(EV_HIST);
@@ -760,6 +793,11 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     if (e == cudaSuccess)
       e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
                               (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true);
+    if (e == cudaSuccess && g.phase2_copy) {
+      // the planner's row copies of Phase 2 wait for the permuted rows
+      e = cudaEventRecord(c->ev_gather, st);
+      c->gather_seq.store(seq, std::memory_order_release);
+    }
     if (e != cudaSuccess) rc = fail(c, FEPLB_E_CUDA, "dispatch launch: %s", cudaGetErrorString(e));
   }
   TL_EVENT(EV_DISPATCH);

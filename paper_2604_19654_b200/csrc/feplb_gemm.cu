@@ -230,7 +230,8 @@ __device__ __forceinline__ void warp_scan_prefix(SmemTail* t, int first, int n, 
 
 template <bool SWIGLU, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
-k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_ra,
+               const __grid_constant__ CUtensorMap tm_b0,
                const __grid_constant__ CUtensorMap tm_b1, const __grid_constant__ CUtensorMap tm_r0,
                const __grid_constant__ CUtensorMap tm_r1, const __grid_constant__ CUtensorMap tm_out, const GemmParams p) {
   constexpr int kStages = Ring<PAIR>::kStages, kStageBytes = Ring<PAIR>::kStageBytes;
@@ -254,6 +255,7 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   // ---- set-up: barriers, TMEM, group table ------------------------------------------------
   if (threadIdx.x == 0) {
     prefetch_tmap(&tm_a);
+    prefetch_tmap(&tm_ra);
     prefetch_tmap(&tm_b0);
     prefetch_tmap(&tm_b1);
     prefetch_tmap(&tm_r0);
@@ -368,7 +370,9 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       unsigned long long peek = 0;
       if (!dyn_known && lane == 0) peek = ld_relaxed_gpu_u64(p.dyn.ready_dev);
       if (lane == 0) {
-        // weights of a migrated expert come from its slot of the receive buffer
+        // weights of a migrated expert come from its slot of the receive buffer, and in pass 1 its
+        // rows from the receive region of the rows (same row numbers as the permuted buffer)
+        const CUtensorMap* ma = c.slot >= 0 ? &tm_ra : &tm_a;
         const CUtensorMap* mb0 = c.slot >= 0 ? &tm_r0 : &tm_b0;
         const CUtensorMap* mb1 = c.slot >= 0 ? &tm_r1 : &tm_b1;
         const int brow0 = (c.slot >= 0 ? c.slot : c.expert) * p.b_rows_per_expert + (SWIGLU ? c.nt * p.bn : c.nt * 2 * p.bn);
@@ -387,12 +391,12 @@ k_grouped_gemm(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t full0 = map_to_cta(full, 0);
             const bool peer_rows = c.rows_valid > BM;
             if (cta_rank == 0) mbar_expect_tx(full, peer_rows ? stage_tx : stage_tx - kABytes);
-            if (cta_rank == 0 || peer_rows) tma_load_2d_pair(sa, &tm_a, full0, kb * BK, c.row0 + (int)cta_rank * BM);
+            if (cta_rank == 0 || peer_rows) tma_load_2d_pair(sa, ma, full0, kb * BK, c.row0 + (int)cta_rank * BM);
             if (cta_rank == 0) tma_load_2d_pair(sb, mb0, full0, kb * BK, brow0);
             else tma_load_2d_pair(sb, mb1, full0, kb * BK, brow1);
           } else {
             mbar_expect_tx(full, stage_tx);
-            tma_load_2d(sa, &tm_a, full, kb * BK, c.row0);
+            tma_load_2d(sa, ma, full, kb * BK, c.row0);
             tma_load_2d(sb, mb0, full, kb * BK, brow0);
             tma_load_2d(sb + b_half_bytes, mb1, full, kb * BK, brow1);
           }
@@ -595,7 +599,7 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t inner, 
 }
 
 template <bool SWIGLU, bool PAIR>
-cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tr0,
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tra, const CUtensorMap& tb0, const CUtensorMap& tb1, const CUtensorMap& tr0,
                        const CUtensorMap& tr1, const CUtensorMap& tout, const GemmParams& p, int num_sms, cudaStream_t st) {
   // per instantiation and device: the shared-memory attribute and the resident grid are set on first use
   static int grid_of[64] = {};
@@ -635,7 +639,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb0, const CUte
     grid = g;
   }
   cfg.gridDim = dim3(grid);
-  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tb0, tb1, tr0, tr1, tout, p);
+  return cudaLaunchKernelEx(&cfg, k_grouped_gemm<SWIGLU, PAIR>, ta, tra, tb0, tb1, tr0, tr1, tout, p);
 }
 
 }  // namespace
@@ -671,6 +675,12 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
     snprintf(err, errn, "cuTensorMapEncodeTiled failed for the receive buffer");
     return FEPLB_E_CUDA;
   }
+  // rows of migrated pieces: pass 1 reads them from the receive region when there is one
+  CUtensorMap tm_rx = tm_x;
+  if (has_recv && a.recv_x && !make_tmap(&tm_rx, a.recv_x, (uint64_t)a.s_cap, (uint64_t)a.d, BM)) {
+    snprintf(err, errn, "cuTensorMapEncodeTiled failed for the receive region of the rows");
+    return FEPLB_E_CUDA;
+  }
   GemmParams p1;
   p1.n_recv_slots = has_recv ? a.n_recv_slots : 0;
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which; p1.E = a.E; p1.s_cap = a.s_cap;
@@ -684,12 +694,12 @@ int feplb_launch_expert_ffn(const feplb_gemm_args& a, cudaStream_t st, int64_t* 
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d; p2.ab_out = nullptr;
   p2.stamps = p1.stamps ? p1.stamps + 4 : nullptr;
 
-  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st)
-                         : launch_one<true, false>(tm_x, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st);
+  cudaError_t e = a.pair ? launch_one<true, true>(tm_x, tm_rx, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st)
+                         : launch_one<true, false>(tm_x, tm_rx, tm_w1, tm_w3, tm_r1, tm_r3, tm_ho, p1, a.num_sms, st);
   ++*n_launch;
   if (e == cudaSuccess) {
-    e = a.pair ? launch_one<false, true>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st)
-               : launch_one<false, false>(tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st);
+    e = a.pair ? launch_one<false, true>(tm_h, tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st)
+               : launch_one<false, false>(tm_h, tm_h, tm_w2, tm_w2, tm_r2, tm_r2, tm_yo, p2, a.num_sms, st);
     ++*n_launch;
   }
   if (e != cudaSuccess) {

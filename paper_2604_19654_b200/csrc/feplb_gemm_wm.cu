@@ -202,7 +202,7 @@ template <bool SWIGLU>
 __global__ void __launch_bounds__(kThreads, 1)
 k_ffn_wm(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ CUtensorMap tm_a1,
          const __grid_constant__ CUtensorMap tm_r0, const __grid_constant__ CUtensorMap tm_r1,
-         const __grid_constant__ BMaps tm_b, const WmParams p) {
+         const __grid_constant__ BMaps tm_b, const __grid_constant__ BMaps tm_rb, const WmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* epi_smem = smem + (size_t)kRingBytes;
@@ -352,7 +352,7 @@ k_ffn_wm(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ CUte
           } else {
             tma_load_2d_pair(sa, ma0, full, kb * BK, arow0);                  // 128 rows of W2
           }
-          tma_load_2d_pair(sa + kATile, &tm_b.m[bi], full, kb * BK, brow0);
+          tma_load_2d_pair(sa + kATile, c.slot >= 0 ? &tm_rb.m[bi] : &tm_b.m[bi], full, kb * BK, brow0);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -552,7 +552,7 @@ bool make_bmaps(BMaps* b, const void* base, uint64_t rows, uint64_t inner) {
 
 template <bool SWIGLU>
 cudaError_t launch_wm(const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& r0, const CUtensorMap& r1,
-                      const BMaps& b, const WmParams& p, int num_sms, cudaStream_t st) {
+                      const BMaps& b, const BMaps& rb, const WmParams& p, int num_sms, cudaStream_t st) {
   // per instantiation and device: the shared-memory attribute and the resident grid are set on first use
   static int grid_of[64] = {};
   int dev = 0;
@@ -583,7 +583,7 @@ cudaError_t launch_wm(const CUtensorMap& a0, const CUtensorMap& a1, const CUtens
     grid = 2 * (n_clusters < num_sms / 2 ? n_clusters : num_sms / 2);
   }
   cfg.gridDim = dim3(grid);
-  return cudaLaunchKernelEx(&cfg, k_ffn_wm<SWIGLU>, a0, a1, r0, r1, b, p);
+  return cudaLaunchKernelEx(&cfg, k_ffn_wm<SWIGLU>, a0, a1, r0, r1, b, rb, p);
 }
 
 }  // namespace
@@ -617,6 +617,11 @@ int feplb_launch_expert_ffn_wm(const feplb_gemm_args& a, const feplb_wm_dyn& dyn
     snprintf(err, errn, "cuTensorMapEncodeTiled failed for the receive buffer");
     return FEPLB_E_CUDA;
   }
+  BMaps brx = bx;      // rows of migrated pieces: pass 1 reads them from the receive region when there is one
+  if (has_recv && a.recv_x && !make_bmaps(&brx, a.recv_x, (uint64_t)a.s_cap, (uint64_t)a.d)) {
+    snprintf(err, errn, "cuTensorMapEncodeTiled failed for the receive region of the rows");
+    return FEPLB_E_CUDA;
+  }
   WmParams p1;
   p1.groups = a.groups; p1.n_groups = a.n_groups; p1.which = a.which;
   p1.dyn = feplb_dyn_table(dyn);
@@ -632,10 +637,10 @@ int feplb_launch_expert_ffn_wm(const feplb_gemm_args& a, const feplb_wm_dyn& dyn
   p2.out = (__nv_bfloat16*)a.y; p2.ld_out = a.d; p2.ab_out = nullptr;
   p2.stamps = dyn.stamps ? dyn.stamps + 4 : nullptr;
 
-  cudaError_t e = launch_wm<true>(tm_w1, tm_w3, tm_r1, tm_r3, bx, p1, a.num_sms, st);
+  cudaError_t e = launch_wm<true>(tm_w1, tm_w3, tm_r1, tm_r3, bx, brx, p1, a.num_sms, st);
   ++*n_launch;
   if (e == cudaSuccess) {
-    e = launch_wm<false>(tm_w2, tm_w2, tm_r2, tm_r2, bh, p2, a.num_sms, st);
+    e = launch_wm<false>(tm_w2, tm_w2, tm_r2, tm_r2, bh, bh, p2, a.num_sms, st);
     ++*n_launch;
   }
   if (e != cudaSuccess) {

@@ -72,6 +72,7 @@ struct feplb_gemm_args {
   int pair;   // 1: clusters of two CTAs on 256-row tiles (cta_group::2); 0: one CTA per 128-row tile
   // receive buffer of migrated experts' weights ([n_recv_slots, f, d] x2 and [n_recv_slots, d, f]); may be null
   const void* recv_w1; const void* recv_w3; const void* recv_w2; int n_recv_slots;
+  const void* recv_x = nullptr;   // optional [s_cap, d]: rows of pieces that run from a receive slot are read here (pass 1)
   void* ab_out;   // optional [s_cap, 2f]: pass 1 also saves the pre-activations a | b (for the backward pass)
 };
 // Returns FEPLB_OK or a feplb_status; text of a failure goes to err (size errn).

@@ -114,7 +114,7 @@ def test_cfg3_full_size_with_phase2_weight_copies(cfg3_weights):
     case.ctx.set_timeline(True)
     p = _check_full_size(case, n_experts=6, n_tokens=8)
     tl = case.ctx.get_timeline()
-    assert tl["phase2_copy_bytes"] == 3 * 6144 * 2048 * 2 * len(p.moves)
+    assert tl["phase2_copy_bytes"] == 3 * 6144 * 2048 * 2 * len(p.moves) + sum(m[3] for m in p.moves) * 6144 * 2   # weights and rows
     case.close()
 
 

@@ -680,7 +680,8 @@ def test_phase2_weight_copies_leave_the_output_unchanged(name, kw):
     assert p1.moves == p0.moves and p1.groups == p0.groups and len(p1.moves) >= 1
     assert np.array_equal(F.bf16_bits(case.buf.out), out0)
     tl = case.ctx.get_timeline()
-    assert tl["phase2_copy_bytes"] == 3 * w.d * w.f * 2 * len(p1.moves)
+    moved_rows = sum(m[3] for m in p1.moves)
+    assert tl["phase2_copy_bytes"] == 3 * w.d * w.f * 2 * len(p1.moves) + moved_rows * w.d * 2     # weights and rows
     assert tl["dev_counts_to_copies_done_us"] > 0
 
     # the kernel reads a migrated piece's weights from its receive slot, not from the home arrays:
@@ -699,6 +700,17 @@ def test_phase2_weight_copies_leave_the_output_unchanged(name, kw):
     assert torch.equal(case.buf.y_perm[grp[1]: grp[1] + grp[2]].view(torch.int16), y_ref.view(torch.int16))
     d_groups = upload_groups([(e, grp[1], grp[2], dst, 1)])        # labelled "home weights": zeros in, zeros out
     case.ctx.expert_ffn(case.buf.x_perm, zero1, zero1, zero2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
+    torch.cuda.synchronize()
+    assert not case.buf.y_perm[grp[1]: grp[1] + grp[2]].float().abs().max().item()
+    # ... and the piece's ROWS from the receive region of the rows, not from the permuted buffer: with the
+    # piece's rows of x_perm zeroed the slot label still gives the same y, the home label gives zeros
+    case.buf.x_perm[grp[1]: grp[1] + grp[2]] = 0
+    d_groups = upload_groups([(e, grp[1], grp[2], dst, 2 + slot)])
+    case.ctx.expert_ffn(case.buf.x_perm, case.d_w1, case.d_w3, case.d_w2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
+    case.ctx.check_status()
+    assert torch.equal(case.buf.y_perm[grp[1]: grp[1] + grp[2]].view(torch.int16), y_ref.view(torch.int16))
+    d_groups = upload_groups([(e, grp[1], grp[2], dst, 1)])
+    case.ctx.expert_ffn(case.buf.x_perm, case.d_w1, case.d_w3, case.d_w2, d_groups, 1, case.buf.h_scratch, case.buf.y_perm)
     torch.cuda.synchronize()
     assert not case.buf.y_perm[grp[1]: grp[1] + grp[2]].float().abs().max().item()
     # a slot beyond the receive buffer is reported, not dereferenced
