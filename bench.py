@@ -312,7 +312,7 @@ def run_cuda(args, w):
         strag = measure_stragglers(F, ctx, w, cfg, buf, dev, d_w1, d_w3, d_w2, stream, n_mb)
     args.backward_result = None
     if rank == 0 and args.backward:
-        args.backward_result = measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, min(args.steps, 100))
+        args.backward_result = measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, min(args.steps, 100), args.bwd_pair)
     _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals, n_fw, e2e_value, h2d, d2h, strag, weights, n_mb)
     ctx.close()
     if world > 1:
@@ -464,12 +464,13 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
-def measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, steps):
+def measure_backward(F, w, dev, d_w1, d_w3, d_w2, stream, n_mb, steps, bwd_pair=-1):
     """Forward + backward of the layer (weight gradients included, so expert segments are padded
     to 128 rows), timed per phase with CUDA events on the launching stream."""
     import torch
     cfg = F.config_from_workload(w, row_align=128)
     ctx, buf, bwd = F.Context(cfg), F.Buffers(cfg), F.BackwardBuffers(cfg)
+    ctx.set_gemm_form(F.FORM_AUTO, bwd_pair)
     ctx.set_preact_buffer(bwd.ab)
     w1t = torch.empty(w.E, w.d, w.f, dtype=torch.bfloat16, device="cuda")
     w3t = torch.empty_like(w1t)
@@ -637,6 +638,10 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
                 "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
                 "traffic": traffic["bytes"] if traffic else None, "traffic_source": traffic["source"] if traffic else None,
                 "launches_timed": gemm_launches, "avg_launch_us": ffn_us / gemm_launches if gemm_launches else None,
+                # the same launches by the GPU's own timer (first CTA's start to last CTA's end, taken inside
+                # the kernels; merged launches only): without the launch gap the CUDA events include
+                "avg_launch_us_kernel_timer": ((totals["dev_ffn_pass1_us"] + totals["dev_ffn_pass2_us"]) / gemm_launches
+                                               if gemm_launches and totals.get("dev_ffn_pass1_us") else None),
                 "dispatch_gbs": io_bytes / (totals["dev_dispatch_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_dispatch_us"] else None,
                 "combine_gbs": io_bytes / (totals["dev_combine_us"] / n_fw * 1e-6) / 1e9 if n_fw and totals["dev_combine_us"] else None,
                 "dispatch_gbs_cold": cold.get("dispatch_gbs_cold"), "combine_gbs_cold": cold.get("combine_gbs_cold"),
@@ -646,7 +651,8 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
         targets = None
         if achieved:
             hbm = peaks["hbm_gbs"]
-            targets = {"gemm_ge_0.60_of_burst_bf16_peak": bool(achieved / peaks["bf16_tflops"] >= 0.60),
+            targets = {"gemm_ge_0.60_of_bf16_peak_of_this_clock_regime": bool(achieved / peak >= 0.60),
+                       "gemm_ge_0.60_of_burst_bf16_peak": bool(achieved / peaks["bf16_tflops"] >= 0.60),
                        "dispatch_ge_0.60_of_hbm_peak": bool(roof["dispatch_gbs"] and roof["dispatch_gbs"] / hbm >= 0.60),
                        "combine_ge_0.60_of_hbm_peak": bool(roof["combine_gbs"] and roof["combine_gbs"] / hbm >= 0.60),
                        "dispatch_cold_ge_0.60_of_hbm_peak": bool(cold.get("dispatch_gbs_cold", 0) / hbm >= 0.60) if cold else None,
@@ -756,6 +762,8 @@ def main():
                     help="grouped-GEMM form of the forward launches (feplb_set_gemm_form); auto is the library's choice")
     ap.add_argument("--merge", type=int, default=-1, choices=[-1, 0, 1],
                     help="feplb_set_launch_merging: 1 = one GEMM launch per pass over static then dynamic groups, 0 = four launches, -1 = library's choice")
+    ap.add_argument("--bwd-pair", type=int, default=-1, choices=[-1, 0, 1, 2, 3],
+                    help="with --backward: pair mask of the backward GEMMs (feplb_set_gemm_form), -1 = library's choice")
     ap.add_argument("--quick", action="store_true",
                     help="device-resident timing only: no end-to-end loop, stragglers or CPU baseline (for profiling)")
     ap.add_argument("--sweep", default=None,

@@ -530,7 +530,7 @@ static int dispatch_impl(feplb_ctx* c, const void* x, const int32_t* topk_ids, c
   CUDA_TRY(c, feplb_launch_permute(topk_ids, S, g.K, g.E, g.row_align, counts, c->d_block_hist, c->d_pad_off,
                                    slot_to_row, row_to_token, (int64_t)c->s_cap, c->d_status, st, &c->launches));
   CUDA_TRY(c, feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
-                                  (int64_t)c->s_cap, c->num_sms, st, &c->launches));
+                                  (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true));
   return FEPLB_OK;
 }
 
@@ -684,9 +684,10 @@ static int harvest_slot(feplb_ctx* c, int r) {
   feplb_timeline t = c->ev_host[r];
   t.dev_hist_us = el(ev[EV_T0], ev[EV_HIST]);
   t.dev_dispatch_us = el(ev[EV_HIST], ev[EV_DISPATCH]);
+  const bool merged = t.ffn_launches == 2;
   t.dev_static_ffn_us = el(ev[EV_STATIC0], ev[EV_STATIC1]);
-  t.dev_dynamic_ffn_us = el(ev[EV_DYN0], ev[EV_DYN1]);
-  t.dev_combine_us = el(ev[EV_DYN1], ev[EV_COMBINE]);
+  t.dev_dynamic_ffn_us = merged ? 0.0 : el(ev[EV_DYN0], ev[EV_DYN1]);
+  t.dev_combine_us = el(ev[merged ? EV_STATIC1 : EV_DYN1], ev[EV_COMBINE]);
   t.dev_counts_to_static_start_us = el(ev[EV_COUNTS], ev[EV_STATIC0]);
   t.dev_counts_to_static_end_us = el(ev[EV_COUNTS], ev[EV_STATIC1]);
   t.dev_total_us = el(ev[EV_T0], ev[EV_COMBINE]);
@@ -814,10 +815,8 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
     if (rc == FEPLB_OK)
       rc = ffn_impl(c, x_perm, w1, w3, w2, c->d_home_groups, g.E, FEPLB_FFN_STATIC, h_scratch, y_perm, st,
                     c->gemm_pair_forced >= 0 ? c->gemm_pair_forced : (int)c->merged_pair, &dyn);
-    TL_EVENT(EV_STATIC1);
+    TL_EVENT(EV_STATIC1);          // both launches lie between EV_STATIC0 and here; no events of their own for the dynamic part
     c->tl.host_enqueue_static_done_us = us_since(c->t0);
-    TL_EVENT(EV_DYN0);
-    TL_EVENT(EV_DYN1);
     int rc_comb = rc == FEPLB_OK ? feplb_combine(c, y_perm, slot_to_row, gates, out, stream) : FEPLB_OK;
     if (c->timeline_on && rc == FEPLB_OK && rc_comb == FEPLB_OK) {
       cudaError_t e = cudaEventRecord(c->ev[EV_COMBINE], st);

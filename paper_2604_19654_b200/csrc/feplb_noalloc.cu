@@ -86,7 +86,7 @@ extern "C" int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, co
                            row_to_token, s_cap, st_word, st, &launches) != cudaSuccess)
     return FEPLB_E_CUDA;
   if (feplb_launch_gather(x, slot_to_row, counts, pad_off, x_perm, cfg->T, cfg->K, cfg->E, cfg->d, cfg->row_align,
-                          s_cap, num_sms, st, &launches) != cudaSuccess)
+                          s_cap, num_sms, st, &launches, row_to_token, true) != cudaSuccess)
     return FEPLB_E_CUDA;
   return FEPLB_OK;
 }

@@ -126,10 +126,11 @@ __device__ __forceinline__ V block_exclusive_scan(V v, V* tmp, V* total) {
 // k_rank then drops the rows that do not fit.
 __global__ void __launch_bounds__(1024)
 k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __restrict__ counts,
-       int32_t* __restrict__ pad_off, int64_t s_cap, uint32_t* status) {
+       int32_t* __restrict__ pad_off, int64_t s_cap, uint32_t* status, int32_t* __restrict__ row_to_token) {
   __shared__ long long tmp[64];
   const int e = threadIdx.x;
   int c = 0;
+  pdl_sync();
   if (e < E) {
     int run = 0;
     for (int b = 0; b < nb; ++b) {
@@ -148,6 +149,9 @@ k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __
     pad_off[E] = (int32_t)(total < s_cap ? total : s_cap);
     if (total > s_cap) atomicOr(status, FEPLB_ST_COUNTS);
   }
+  // rows behind the last segment hold no token (the padding rows inside segments are marked by k_zero_pad,
+  // the live rows by k_rank: with counts that agree with the ids that covers every row)
+  for (int64_t i = total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
 }
 
 // Whole-layer variant of k_scan: from the per-CTA histograms alone it produces everything the
@@ -429,21 +433,23 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
                                  int32_t* block_hist, int32_t* pad_off, int32_t* slot_to_row,
                                  int32_t* row_to_token, int64_t s_cap, uint32_t* status,
                                  cudaStream_t st, int64_t* n_launch) {
+  // three kernels chained by programmatic launches (each one's launch latency hides under its predecessor)
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
-  if (s_cap > 0 && (err = cudaMemsetAsync(row_to_token, 0xFF, sizeof(int32_t) * s_cap, st)) != cudaSuccess) return err;
   if (nb) {
-    k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E, block_hist, nullptr, nullptr, status);
+    err = launch(k_block_hist, nb, kThreads, sizeof(int) * kWarps * E, st, false, ids, S, E, E, block_hist,
+                 (int32_t*)nullptr, (int32_t*)nullptr, status);
     ++*n_launch;
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    if (err != cudaSuccess) return err;
   }
-  k_scan<<<1, 1024, 0, st>>>(block_hist, nb, E, A, counts, pad_off, s_cap, status);
+  err = launch(k_scan, 1, 1024, 0, st, nb > 0, block_hist, nb, E, A, counts, pad_off, s_cap, status, row_to_token);
   ++*n_launch;
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if (err != cudaSuccess) return err;
   if (nb) {
-    k_rank<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, K, E, block_hist, pad_off, slot_to_row, row_to_token, s_cap);
+    err = launch(k_rank, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, K, E, (const int32_t*)block_hist,
+                 (const int32_t*)pad_off, slot_to_row, row_to_token, s_cap);
     ++*n_launch;
-    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    if (err != cudaSuccess) return err;
   }
   return cudaSuccess;
 }
