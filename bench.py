@@ -30,9 +30,11 @@ from paper_2604_19654_b200 import workloads as W  # noqa: E402
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 # DRAM bytes (read + write) of one k_grouped_gemm launch at the benchmarked workload, from the ncu
-# capture summarised under profiles/; None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "cfg2": {"bytes": 190.0e6, "source": "profiles/k_grouped_gemm_cfg2.md: 760 MB over the 4 launches of one forward"},
+# capture summarised under profiles/; none (null in the line) where no capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {     # keyed by (workload, GEMM launches per forward)
+    ("cfg2", 2): {"bytes": 380.3e6, "source": "profiles/k_grouped_gemm_cfg2.md: 760.6 MB over the 2 launches of one forward "
+                                              "(capture of the merged two-CTA launches)"},
+    ("cfg2", 4): {"bytes": 190.0e6, "source": "capture of the four-launch form: 760 MB over the 4 launches of one forward"},
 }
 
 
@@ -627,7 +629,7 @@ def _report(args, w, ctx, rank, world, value, ms_total, launches, clocks, totals
         sus = peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]
         io_bytes = 2.0 * (w.T * w.d + w.S * w.d) + 12.0 * w.S
         cold = getattr(args, "cold", None) or {}
-        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(w.name)
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((w.name, per_fw)) if args.form in ("auto", "pair") else None
         roof = {"bound": "tensor", "kernel": ("k_grouped_gemm, static + dynamic groups per launch" if per_fw == 2 else "k_grouped_gemm") if args.form != "weight_m" else "k_ffn_wm",
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak if achieved else None,
