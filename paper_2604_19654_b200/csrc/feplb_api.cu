@@ -529,8 +529,8 @@ static int dispatch_impl(feplb_ctx* c, const void* x, const int32_t* topk_ids, c
   }
   CUDA_TRY(c, feplb_launch_permute(topk_ids, S, g.K, g.E, g.row_align, counts, c->d_block_hist, c->d_pad_off,
                                    slot_to_row, row_to_token, (int64_t)c->s_cap, c->d_status, st, &c->launches));
-  CUDA_TRY(c, feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
-                                  (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true));
+  CUDA_TRY(c, feplb_launch_gather(x, topk_ids, c->d_block_hist, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E,
+                                  g.d, g.row_align, (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true));
   return FEPLB_OK;
 }
 
@@ -778,7 +778,7 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   c->flag_seq = c->flag_seq == INT32_MAX ? 1 : c->flag_seq + 1;
   const int32_t seq = c->flag_seq;
   CUDA_TRY(c, feplb_launch_route_fused(topk_ids, S, g.E, g.R, g.row_align, g.dyn, mask_dev, c->d_block_hist, counts,
-                                       rank_load, c->d_pad_off, c->d_home_groups, nullptr, row_to_token,
+                                       rank_load, c->d_pad_off, c->d_home_groups, nullptr, slot_to_row, row_to_token,
                                        (int64_t)c->s_cap, c->d_status, c->h_counts_tagged, seq,
                                        stamps ? stamps + 8 : nullptr, st, &c->launches));
   c->job_w1 = w1; c->job_w3 = w3; c->job_w2 = w2;   // read by the planner thread after it is woken
@@ -789,11 +789,9 @@ extern "C" int feplb_moe_forward(feplb_ctx* c, const void* x, const int32_t* top
   // step 3: permutation (does not depend on the plan: a migration relabels rows, it does not move
   // them here).  From here on a failure must still join the planner, so errors are carried in rc.
   {
-    cudaError_t e = feplb_launch_rank(topk_ids, S, g.K, g.E, c->d_block_hist, c->d_pad_off, slot_to_row, row_to_token,
-                                      (int64_t)c->s_cap, st, &c->launches);
-    if (e == cudaSuccess)
-      e = feplb_launch_gather(x, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K, g.E, g.d, g.row_align,
-                              (int64_t)c->s_cap, c->num_sms, st, &c->launches, row_to_token, true);
+    cudaError_t e = feplb_launch_gather(x, topk_ids, c->d_block_hist, slot_to_row, counts, c->d_pad_off, x_perm, g.T, g.K,
+                                        g.E, g.d, g.row_align, (int64_t)c->s_cap, c->num_sms, st, &c->launches,
+                                        row_to_token, true);
     if (e == cudaSuccess && g.phase2_copy) {
       // the planner's row copies of Phase 2 wait for the permuted rows
       e = cudaEventRecord(c->ev_gather, st);

