@@ -359,7 +359,7 @@ def measure_cold_io(F, ctx, cfg, w, dev, stream, reps=24):
             "dispatch_us": float(np.median(t_disp)) * 1e3, "combine_us": float(np.median(t_comb)) * 1e3,
             "dispatch_gbs_cold": io_bytes / (float(np.median(t_disp)) * 1e-3) / 1e9,
             "combine_gbs_cold": io_bytes / (float(np.median(t_comb)) * 1e-3) / 1e9,
-            "note": "stand-alone feplb_dispatch (histogram, scan, ranking, gather) and feplb_combine, one call per "
+            "note": "stand-alone feplb_dispatch (histogram + ranks, scan, gather) and feplb_combine, one call per "
                     "buffer set in rotation; the in-pipeline (warm) figures are roofline.dispatch_gbs / combine_gbs"}
 
 

@@ -299,10 +299,10 @@ k_gather(const uint4* __restrict__ x, const int32_t* __restrict__ ids, const int
       if (lane < K) {
         const int64_t s = (int64_t)t * K + lane;
         const int r = __ldcg(slot_to_row + s);
+        const int e = ids[s];    // in flight together with r; its offsets follow in one more round trip
         if (r >= 0) {
           myrow = r;             // already final
-        } else if (r <= -2) {
-          const int e = ids[s];
+        } else if (r <= -2) {    // implies 0 <= e < E (checked by k_block_hist)
           const int64_t row = (int64_t)pad_off[e] + block_base[s / FEPLB_SLOTS_PER_BLOCK * E + e] + (-2 - r);
           // rows beyond the buffer: only with counts that disagree with the ids (reported by the scan)
           myrow = row < s_cap ? (int)row : -1;
