@@ -33,7 +33,9 @@ def _tiny(T, K, E, R, d=128, f=64, **kw):
 
 HIST_CASES = [W.get_workload("cfg1"), W.get_workload("cfg2"), W.get_workload("cfg4"),
               _tiny(1, 1, 4, 2), _tiny(37, 3, 6, 3), _tiny(1025, 5, 16, 4), _tiny(3000, 8, 128, 8),
-              _tiny(64, 2, 1, 1)]
+              _tiny(64, 2, 1, 1),
+              _tiny(77, 8, 16, 4, d=6144),       # six 2 KiB slices per row: a token's slices are copied by several warps and CTAs
+              _tiny(50, 32, 64, 4, d=256)]       # the largest top-k
 
 
 @pytest.mark.parametrize("w", HIST_CASES, ids=lambda w: f"{w.name}-T{w.T}K{w.K}E{w.E}")
@@ -80,6 +82,42 @@ def test_out_of_range_expert_id_is_reported_not_trapped():
     assert ei.value.code == F.E_RANGE
     assert int(buf.counts.sum()) == w.T * w.K - 2
     ctx.check_status()                                                    # the status word was cleared
+    ctx.close()
+
+
+def test_dispatch_skips_slots_with_an_id_out_of_range():
+    """Slots whose id lies outside [0, E) get slot_to_row = -1 and no row; every other slot is ranked as the
+    stable counting sort over the valid slots alone ranks it, and the error is reported."""
+    torch = _torch()
+    w = _tiny(300, 4, 8, 2, d=2304)                                       # 2304 / 8 = 288 chunks: a ragged third slice
+    cfg = F.config_from_workload(w)
+    ctx, buf = F.Context(cfg), F.Buffers(cfg)
+    rng = np.random.default_rng(5)
+    ids = rng.integers(0, w.E, size=(w.T, w.K)).astype(np.int32)
+    bad = rng.random(ids.shape) < 0.05
+    ids[bad] = np.where(rng.random(bad.sum()) < 0.5, w.E + 3, -1)
+    x = W.gen_activations(w, 0)
+    d_ids = torch.from_numpy(ids).cuda()
+    ctx.route_hist(d_ids, buf.counts, buf.rank_load)
+    with pytest.raises(F.FeplbError):
+        ctx.check_status()
+    buf.x_perm.fill_(7.0)
+    ctx.dispatch(F.bf16_tensor(x), d_ids, buf.counts, buf.x_perm, buf.slot_to_row, buf.row_to_token)
+    with pytest.raises(F.FeplbError) as ei:
+        ctx.check_status()
+    assert ei.value.code == F.E_RANGE
+    flat = ids.reshape(-1)
+    valid = np.flatnonzero(~bad.reshape(-1))
+    order = valid[np.argsort(flat[valid], kind="stable")]                 # valid slots in expert order, ties by slot
+    want = np.full(flat.size, -1, np.int32)
+    want[order] = np.arange(order.size, dtype=np.int32)
+    assert np.array_equal(buf.slot_to_row.cpu().numpy().reshape(-1), want)
+    r2t = buf.row_to_token.cpu().numpy()
+    assert np.array_equal(r2t[: order.size], (order // w.K).astype(np.int32))
+    assert np.all(r2t[order.size:] == -1)
+    got = F.bf16_bits(buf.x_perm)
+    assert np.array_equal(got[: order.size], x[order // w.K])
+    assert np.all(got[order.size:] == 0x40E0)                             # bf16 7.0: rows without a slot stay untouched
     ctx.close()
 
 
