@@ -154,17 +154,18 @@ def test_plan_upload_lands_inside_the_static_window(name, cfg3_weights):
         case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf, want_plan=False)
     case.ctx.check_status()
     case.ctx.set_timeline(True)
-    host, dev = [], []
+    host, dev, plan_us = [], [], []
     for _ in range(20):
         case.ctx.moe_forward(case.d_x, case.d_ids, case.d_gates, case.d_w1, case.d_w3, case.d_w2, case.buf, want_plan=False)
         tl = case.ctx.get_timeline()
         host.append(tl["host_upload_enqueued_us"] - tl["host_counts_ready_us"])
         dev.append(tl["dev_counts_to_static_end_us"])
+        plan_us.append(tl["plan_us"])
     case.ctx.check_status()
     assert min(host) >= 0 and min(dev) > 0
     assert np.median(host) < np.median(dev), (np.median(host), np.median(dev))
     # the greedy itself is tens of microseconds at most (the paper quotes ~50 us on one core)
-    assert tl["plan_us"] < 200
+    assert np.median(plan_us) < 200
     case.close()
 
 
