@@ -63,3 +63,36 @@ def test_activations_and_weights():
     assert not np.array_equal(w1, w3)
     assert np.array_equal(W.gen_weights(w)[2], w2)
     assert len(W.sweep_points()) == 20
+
+
+# ----------------------------------------------------------------------------- bench.py host arithmetic
+
+def test_bench_peak_selection_and_roofline_arithmetic():
+    """The bf16 denominator follows the clock regime of the run; flops per micro-batch are 6 d f per slot; the
+    timeline of a forward is ordered on one axis."""
+    import bench
+    peaks = {"bf16_tflops": 1634.5, "bf16_tflops_sustained": 1377.1}
+    burst = {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0, "reasons": []}
+    capped = {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0, "reasons": ["sw_power_cap"]}
+    slow = {"sm_mhz": 1500.0, "sm_max_mhz": 1965.0, "reasons": []}
+    assert bench.pick_bf16_peak(peaks, burst) == (1634.5, "burst")
+    assert bench.pick_bf16_peak(peaks, capped)[0] == 1377.1
+    assert bench.pick_bf16_peak(peaks, slow)[0] == 1377.1
+    assert bench.pick_bf16_peak(peaks, None)[0] == 1377.1
+    w = W.get_workload("cfg2")
+    assert bench.gemm_flops(w) == 6.0 * 2048 * 768 * 4096 * 6
+    assert bench.whole_job_throughput(2, 10, 4096, 5.0) == 2 * 10 * 4096 / 5e-3
+    assert bench.rank_microbatches(1, 4) == [4, 5, 6, 7]
+    st = {"dev_hist_us": 16.0, "host_counts_ready_us": 300.0, "host_plan_done_us": 302.5, "plan_us": 1.0,
+          "host_upload_enqueued_us": 302.7, "dev_counts_to_static_start_us": 45.0, "dev_counts_to_static_end_us": 110.0,
+          "dev_total_us": 360.0, "dev_combine_us": 28.0, "dev_dispatch_us": 30.0, "dev_static_ffn_us": 280.0,
+          "dev_dynamic_ffn_us": 0.0, "ffn_launches": 2.0, "dev_ffn_pass1_us": 175.0, "dev_ffn_pass2_us": 96.0,
+          "dev_plan_wait_us": 9.0}
+    tl = bench.merged_timeline(st)
+    assert tl and all(len(e) == 3 and e[1] <= e[2] for e in tl)
+    names = [e[0] for e in tl]
+    assert any("plan" in n for n in names) and any("combine" in n for n in names)
+    plan = [e for e in tl if e[0] == "host: greedy plan"][0]
+    static_end = 16.0 + 110.0
+    assert plan[2] < static_end                       # the plan lands inside the static window of this example
+    assert bench.merged_timeline({}) is None
